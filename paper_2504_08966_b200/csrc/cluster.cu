@@ -1,0 +1,548 @@
+// DBDPC (Algorithm 2) and reincorporation (Eq. 8-9): key gather and inverse norms, all-pairs
+// distance tiles with the density and the d <= d_c adjacency fused into their epilogue, density
+// rank, centre selection, tokens-by-centres nearest-centre pass, labels.
+//
+// This file holds the SIMT tile kernels (any element type and key width); the tcgen05 tile
+// kernels for bf16 keys live in gram_umma.cu and share the epilogue arithmetic of common.cuh.
+#include "kernels.cuh"
+
+namespace pact {
+
+__device__ __forceinline__ uint32_t ld_relaxed_u32(const uint32_t *p) {
+  uint32_t v;
+  asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
+template <typename D> __device__ __forceinline__ typename D::rn_t *rn_tok(const ImgDesc &im);
+template <> __device__ __forceinline__ float *rn_tok<DistF>(const ImgDesc &im) { return im.rn; }
+template <> __device__ __forceinline__ double *rn_tok<DistD>(const ImgDesc &im) { return im.rn64; }
+template <typename D> __device__ __forceinline__ typename D::rn_t *rn_kept(const ImgDesc &im);
+template <> __device__ __forceinline__ float *rn_kept<DistF>(const ImgDesc &im) { return im.rnk; }
+template <> __device__ __forceinline__ double *rn_kept<DistD>(const ImgDesc &im) { return im.rnk64; }
+template <typename D> __device__ __forceinline__ typename D::rn_t *rn_cen(const ImgDesc &im);
+template <> __device__ __forceinline__ float *rn_cen<DistF>(const ImgDesc &im) { return im.rnc; }
+template <> __device__ __forceinline__ double *rn_cen<DistD>(const ImgDesc &im) { return im.rnc64; }
+
+// ---- inverse key norms, survivor gather, per-call initialisation -----------------------------
+// grid (ceil(maxN / 8), B), 256 threads, one warp per work item.
+//  all_tokens = 1: item = token i (inverse norm of every token; survivors are copied to Kp[slot])
+//  all_tokens = 0: item = list position r (token kept_idx[r]); only listed rows are touched
+template <typename T>
+__global__ void __launch_bounds__(256) k_keynorm_gather(const __grid_constant__ Batch bt, int all_tokens) {
+  using D = typename DistOf<T>::type;
+  using rn_t = typename D::rn_t;
+  constexpr int V = Vec<T>::N;
+  const ImgDesc &im = bt.img[blockIdx.y];
+  const int lane = threadIdx.x & 31;
+  const int item = blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int q = all_tokens ? 0 : *im.q_ptr;
+  // per-call initialisation of the arrays later kernels accumulate into
+  {
+    const int gt = blockIdx.x * 256 + threadIdx.x, gs = gridDim.x * 256;
+    for (int r = gt; r < im.Np; r += gs) { im.rho_fix[r] = 0ull; im.rank[r] = 0; }
+    for (int wd = gt; wd < im.Wp; wd += gs) { im.cmask[wd] = 0u; im.rmask[wd] = 0u; }
+    for (int i = gt; i < im.N; i += gs) {
+      im.best[i] = kBestInit;
+      if (!all_tokens) {
+        im.label[i] = -1;
+        if (im.label_user) im.label_user[i] = -1;
+      }
+    }
+  }
+  int i, r;
+  if (all_tokens) {
+    i = item;
+    if (i >= im.N) return;
+    r = im.slot[i];
+  } else {
+    r = item;
+    if (r >= q) return;
+    i = im.kept_idx[r];
+  }
+  const T *row = reinterpret_cast<const T *>(im.Kc) + (size_t)i * im.ldKc;
+  const double ss = row_sumsq<T>(row, bt.d_k, lane);
+  const rn_t rn = (rn_t)(1.0 / sqrt(fmax(ss, 1e-40)));
+  if (lane == 0) {
+    rn_tok<D>(im)[i] = rn;
+    if (r >= 0) rn_kept<D>(im)[r] = rn;
+  }
+  if (r >= 0) {
+    T *dst = reinterpret_cast<T *>(im.Kp) + (size_t)r * bt.d_k;
+    for (int v = lane; v * V < bt.d_k; v += 32)
+      reinterpret_cast<uint4 *>(dst)[v] = reinterpret_cast<const uint4 *>(row)[v];
+  }
+}
+
+// centre keys from a list of token indices (reincorporation as a stage of its own)
+template <typename T>
+__global__ void __launch_bounds__(256) k_center_key_gather(const __grid_constant__ Batch bt) {
+  using D = typename DistOf<T>::type;
+  using rn_t = typename D::rn_t;
+  constexpr int V = Vec<T>::N;
+  const ImgDesc &im = bt.img[blockIdx.y];
+  const int lane = threadIdx.x & 31;
+  const int c = blockIdx.x * 8 + (threadIdx.x >> 5);
+  {
+    const int gt = blockIdx.x * 256 + threadIdx.x, gs = gridDim.x * 256;
+    for (int i = gt; i < im.N; i += gs) im.best[i] = kBestInit;
+  }
+  if (c < *im.m_ptr) {                       // inverse norm of the c-th pruned row
+    const int i = im.pruned_idx[c];
+    const double ss = row_sumsq<T>(reinterpret_cast<const T *>(im.Kc) + (size_t)i * im.ldKc, bt.d_k, lane);
+    if (lane == 0) rn_tok<D>(im)[i] = (rn_t)(1.0 / sqrt(fmax(ss, 1e-40)));
+  }
+  if (c >= *im.C_ptr) return;
+  const int i = im.cidx_ptr[c];
+  const T *row = reinterpret_cast<const T *>(im.Kc) + (size_t)i * im.ldKc;
+  const double ss = row_sumsq<T>(row, bt.d_k, lane);
+  if (lane == 0) rn_cen<D>(im)[c] = (rn_t)(1.0 / sqrt(fmax(ss, 1e-40)));
+  T *dst = reinterpret_cast<T *>(im.Kcen) + (size_t)c * bt.d_k;
+  for (int v = lane; v * V < bt.d_k; v += 32)
+    reinterpret_cast<uint4 *>(dst)[v] = reinterpret_cast<const uint4 *>(row)[v];
+}
+
+// ---- 64 x 64 tile of dot products, 256 threads, thread (ty, tx) owns a 4 x 4 block -----------
+constexpr int TS = 64;   // tile side
+constexpr int KC = 32;   // key elements staged per step
+
+template <typename T, typename acc_t, typename RowA, typename RowB>
+__device__ __forceinline__ void tile_dots(RowA rowA, RowB rowB, int d_k, float (*As)[TS + 4],
+                                          float (*Bs)[TS + 4], acc_t (&acc)[4][4]) {
+  constexpr int V = Vec<T>::N;
+  constexpr int VPR = KC / V;                 // vectors per row per step
+  const int t = threadIdx.x, ty = t >> 4, tx = t & 15;
+#pragma unroll
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b) acc[a][b] = (acc_t)0;
+  for (int k0 = 0; k0 < d_k; k0 += KC) {
+    for (int v = t; v < TS * VPR; v += 256) {
+      const int row = v / VPR, kv = (v % VPR) * V;
+      float x[V], y[V];
+      const T *pa = rowA(row), *pb = rowB(row);
+      const bool inb = k0 + kv < d_k;
+      if (pa && inb) load_vec<T>(pa + k0 + kv, x);
+      else {
+#pragma unroll
+        for (int k = 0; k < V; ++k) x[k] = 0.f;
+      }
+      if (pb && inb) load_vec<T>(pb + k0 + kv, y);
+      else {
+#pragma unroll
+        for (int k = 0; k < V; ++k) y[k] = 0.f;
+      }
+#pragma unroll
+      for (int k = 0; k < V; ++k) { As[kv + k][row] = x[k]; Bs[kv + k][row] = y[k]; }
+    }
+    __syncthreads();
+#pragma unroll 8
+    for (int k = 0; k < KC; ++k) {
+      const float4 a4 = *reinterpret_cast<const float4 *>(&As[k][ty * 4]);
+      const float4 b4 = *reinterpret_cast<const float4 *>(&Bs[k][tx * 4]);
+      const float a[4] = {a4.x, a4.y, a4.z, a4.w}, b[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          if (sizeof(acc_t) == 8) acc[i][j] = fma((acc_t)a[i], (acc_t)b[j], acc[i][j]);
+          else acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        }
+    }
+    __syncthreads();
+  }
+}
+
+// ---- Eq. 5-6: all pairs of survivors; density and adjacency in the epilogue --------------------
+// grid (n_ctas, B) persistent over the tiles of the q x q matrix; nothing of it is stored except
+// one bit per pair (d <= d_c) and one integer density per row.
+template <typename T>
+__global__ void __launch_bounds__(256) k_gram_simt(const __grid_constant__ Batch bt) {
+  using D = typename DistOf<T>::type;
+  using acc_t = typename D::acc_t;
+  const ImgDesc &im = bt.img[blockIdx.y];
+  const int q = *im.q_ptr;
+  const int nt = (q + TS - 1) / TS;
+  const int t = threadIdx.x, ty = t >> 4, tx = t & 15;
+  __shared__ __align__(16) float As[KC][TS + 4];
+  __shared__ __align__(16) float Bs[KC][TS + 4];
+  __shared__ unsigned long long rowsum[TS];
+  __shared__ uint32_t adjw[TS][2];
+  const T *Kp = reinterpret_cast<const T *>(im.Kp);
+  const auto *rnk = rn_kept<D>(im);
+  int band = 0;
+  for (int tile = blockIdx.x; tile < nt * nt; tile += gridDim.x) {
+    const int tm = tile / nt, tn = tile % nt;
+    if (t < TS) { rowsum[t] = 0ull; adjw[t][0] = 0u; adjw[t][1] = 0u; }
+    acc_t acc[4][4];
+    tile_dots<T, acc_t>(
+        [&](int r) { const int g = tm * TS + r; return g < q ? Kp + (size_t)g * bt.d_k : (const T *)nullptr; },
+        [&](int r) { const int g = tn * TS + r; return g < q ? Kp + (size_t)g * bt.d_k : (const T *)nullptr; },
+        bt.d_k, As, Bs, acc);
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+      const int gi = tm * TS + ty * 4 + a;
+      if (gi >= q) continue;
+      const auto rni = rnk[gi];
+      unsigned long long s = 0ull;
+      uint32_t bits = 0u;
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        const int gj = tn * TS + tx * 4 + b;
+        if (gj >= q) continue;
+        auto dd = D::dist(acc[a][b], rni, rnk[gj]);
+        if (gi == gj) dd = 0;
+        s += D::term(dd, im);
+        if (D::within(dd, im)) bits |= 1u << b;
+        if (gi < gj && D::in_band(dd, im)) ++band;
+      }
+      atomicAdd(&rowsum[ty * 4 + a], s);
+      if (bits) atomicOr(&adjw[ty * 4 + a][tx >> 3], bits << ((tx & 7) * 4));
+    }
+    __syncthreads();
+    if (t < TS) {
+      const int gi = tm * TS + t;
+      if (gi < q) atomicAdd(&im.rho_fix[gi], rowsum[t]);
+    } else if (t < 3 * TS) {
+      const int r = (t - TS) >> 1, wd = (t - TS) & 1;
+      const int gi = tm * TS + r;
+      if (gi < q) im.adj[(size_t)gi * im.Wp + tn * 2 + wd] = adjw[r][wd];
+    }
+    __syncthreads();
+  }
+  if (band) atomicAdd(&im.cnt[PACT_CNT_BAND_DC], band);
+}
+
+// ---- density rank: rank_i = #{ j : rho_j > rho_i, or rho_j == rho_i and j < i } ------------------
+// grid (n_ctas, B) persistent over 256 x 256 blocks of pairs.
+__global__ void __launch_bounds__(256) k_rank(const __grid_constant__ Batch bt) {
+  const ImgDesc &im = bt.img[blockIdx.y];
+  const int q = *im.q_ptr;
+  const int nb = (q + 255) / 256;
+  const int t = threadIdx.x;
+  __shared__ unsigned long long keys[256];
+  for (int blk = blockIdx.x; blk < nb * nb; blk += gridDim.x) {
+    const int bi = blk / nb, bj = blk % nb;
+    const int j0 = bj * 256;
+    __syncthreads();
+    keys[t] = (j0 + t < q) ? im.rho_fix[j0 + t] : 0ull;
+    __syncthreads();
+    const int i = bi * 256 + t;
+    if (i < q) {
+      const unsigned long long mine = im.rho_fix[i];
+      const int nj = min(256, q - j0);
+      int c = 0;
+      for (int j = 0; j < nj; ++j) {
+        const unsigned long long o = keys[j];
+        c += (o > mine) || (o == mine && (j0 + j) < i);
+      }
+      if (c) atomicAdd(&im.rank[i], c);
+      if (bj == 0) {
+        const float rf = (float)((double)mine * (1.0 / (double)(1u << kRhoShift)));
+        im.rho[i] = rf;
+        if (im.rho_user) im.rho_user[i] = rf;
+      }
+    }
+  }
+}
+
+// ---- centre selection -------------------------------------------------------------------------
+// The sequential loop of Algorithm 2 picks the lexicographically first maximal independent set of
+// the graph {d_ij <= d_c} in density order; that set is unique, so any schedule that only takes
+// final decisions reproduces it (the argument of Appendix D.2).  A row becomes
+//   removed  once an earlier-ranked neighbour is a centre,
+//   a centre once every earlier-ranked neighbour is removed.
+// Both facts are monotone bits, so rows are resolved asynchronously: each warp owns rows, re-reads
+// the two bit masks and decides what it can, until all its rows are decided.  Launched
+// cooperatively so that every CTA is resident; every wait is bounded.
+__global__ void __launch_bounds__(256) k_centers(const __grid_constant__ Batch bt) {
+  const int lane = threadIdx.x & 31;
+  const int nwarps = gridDim.x * 8;
+  const int gw = blockIdx.x * 8 + (threadIdx.x >> 5);
+  int qs[kMaxBatchPerLaunch + 1];
+  qs[0] = 0;
+  for (int b = 0; b < bt.B; ++b) qs[b + 1] = qs[b] + *bt.img[b].q_ptr;
+  const int total = qs[bt.B];
+  // phase 1: keep only the neighbours that come earlier in density order
+  for (int item = gw; item < total; item += nwarps) {
+    int b = 0;
+    while (item >= qs[b + 1]) ++b;
+    const ImgDesc &im = bt.img[b];
+    const int r = item - qs[b], q = qs[b + 1] - qs[b], nw = (q + 31) >> 5;
+    const int myrank = im.rank[r];
+    uint32_t *row = im.adj + (size_t)r * im.Wp;
+    for (int wd = lane; wd < nw; wd += 32) {
+      uint32_t bits = row[wd], out = 0u;
+      while (bits) {
+        const int bpos = __ffs(bits) - 1;
+        bits &= bits - 1;
+        const int j = wd * 32 + bpos;
+        if (j != r && im.rank[j] < myrank) out |= 1u << bpos;
+      }
+      row[wd] = out;
+    }
+  }
+  __syncwarp();
+  // phase 2: resolve
+  int sweeps = 0, pending = 1;
+  while (pending && sweeps < kSpinLimit) {
+    pending = 0;
+    ++sweeps;
+    for (int item = gw; item < total; item += nwarps) {
+      int b = 0;
+      while (item >= qs[b + 1]) ++b;
+      const ImgDesc &im = bt.img[b];
+      const int r = item - qs[b], q = qs[b + 1] - qs[b], nw = (q + 31) >> 5;
+      const uint32_t mybit = 1u << (r & 31);
+      const uint32_t decided = (ld_relaxed_u32(&im.cmask[r >> 5]) | ld_relaxed_u32(&im.rmask[r >> 5])) & mybit;
+      if (decided) continue;
+      const uint32_t *row = im.adj + (size_t)r * im.Wp;
+      bool hit_center = false, alive = false;
+      for (int wd = lane; wd < nw; wd += 32) {
+        const uint32_t e = row[wd];
+        if (e) {
+          hit_center |= (e & ld_relaxed_u32(&im.cmask[wd])) != 0u;
+          alive |= (e & ~ld_relaxed_u32(&im.rmask[wd])) != 0u;
+        }
+      }
+      hit_center = __any_sync(0xffffffffu, hit_center);
+      alive = __any_sync(0xffffffffu, alive);
+      if (hit_center) {
+        if (lane == 0) atomicOr(&im.rmask[r >> 5], mybit);
+      } else if (!alive) {
+        if (lane == 0) atomicOr(&im.cmask[r >> 5], mybit);
+      } else {
+        pending = 1;
+      }
+    }
+  }
+  if (lane == 0 && total > 0) {
+    for (int b = 0; b < bt.B; ++b) {
+      if (pending) atomicMin(&bt.img[b].cnt[PACT_CNT_STATUS], (int)PACT_ERR_TIMEOUT);
+      atomicMax(&bt.img[b].cnt[PACT_CNT_SWEEPS], sweeps);
+    }
+  }
+}
+
+// ---- cluster ids, centre list, centre keys ------------------------------------------------------
+// grid (n_ctas, B), 256 threads; cluster id of a centre = number of centres with a lower index.
+template <typename T>
+__global__ void __launch_bounds__(256) k_centers_finalize(const __grid_constant__ Batch bt) {
+  using D = typename DistOf<T>::type;
+  constexpr int V = Vec<T>::N;
+  const ImgDesc &im = bt.img[blockIdx.y];
+  const int q = *im.q_ptr, nw = (q + 31) >> 5;
+  const int t = threadIdx.x, lane = t & 31, w = t >> 5;
+  extern __shared__ int pref[];            // [nw + 1] exclusive prefix of popcounts
+  __shared__ int wsum[8];
+  __shared__ int carry;
+  if (t == 0) carry = 0;
+  __syncthreads();
+  for (int base = 0; base < nw; base += 256) {
+    const int wd = base + t;
+    const int pc = wd < nw ? __popc(im.cmask[wd]) : 0;
+    int x = pc;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int y = __shfl_up_sync(0xffffffffu, x, o);
+      if (lane >= o) x += y;
+    }
+    if (lane == 31) wsum[w] = x;
+    __syncthreads();
+    int off = carry;
+    for (int k = 0; k < w; ++k) off += wsum[k];
+    if (wd < nw) pref[wd] = off + x - pc;
+    __syncthreads();
+    if (t == 255) carry = off + x;
+    __syncthreads();
+  }
+  const int C = carry;
+  if (blockIdx.x == 0 && t == 0) {
+    im.cnt[PACT_CNT_C] = C;
+    if (im.C_user) *im.C_user = C;
+  }
+  const T *Kp = reinterpret_cast<const T *>(im.Kp);
+  T *Kcen = reinterpret_cast<T *>(im.Kcen);
+  for (int r = blockIdx.x * 8 + w; r < q; r += gridDim.x * 8) {
+    const uint32_t m = im.cmask[r >> 5];
+    if (!((m >> (r & 31)) & 1u)) continue;
+    const int c = pref[r >> 5] + __popc(m & ((1u << (r & 31)) - 1u));
+    if (lane == 0) {
+      im.cid[r] = c;
+      const int tok = im.kept_idx[r];
+      im.center_idx[c] = tok;
+      if (im.center_idx_user) im.center_idx_user[c] = tok;
+      rn_cen<D>(im)[c] = rn_kept<D>(im)[r];
+    }
+    for (int v = lane; v * V < bt.d_k; v += 32)
+      reinterpret_cast<uint4 *>(Kcen + (size_t)c * bt.d_k)[v] =
+          reinterpret_cast<const uint4 *>(Kp + (size_t)r * bt.d_k)[v];
+  }
+}
+
+// ---- nearest centre of every row (Algorithm 2 assignment; Eq. 8 argmin) ---------------------------
+// grid (n_ctas, B) persistent over 64 x 64 tiles of rows x centres; the running minimum of a row
+// is one 64-bit word (distance bits, cluster id) reduced with atomicMin, so ties go to the lower id.
+template <typename T>
+__global__ void __launch_bounds__(256) k_assign_simt(const __grid_constant__ Batch bt, int mode) {
+  using D = typename DistOf<T>::type;
+  using acc_t = typename D::acc_t;
+  const ImgDesc &im = bt.img[blockIdx.y];
+  const int C = *im.C_ptr;
+  const int nrows = mode == ROWS_ALL ? im.N : (mode == ROWS_KEPT_LIST ? *im.q_ptr : *im.m_ptr);
+  const int32_t *list = mode == ROWS_KEPT_LIST ? im.kept_idx : im.pruned_idx;
+  const int ntm = (nrows + TS - 1) / TS, ntn = (C + TS - 1) / TS;
+  const int t = threadIdx.x, ty = t >> 4, tx = t & 15;
+  __shared__ __align__(16) float As[KC][TS + 4];
+  __shared__ __align__(16) float Bs[KC][TS + 4];
+  __shared__ unsigned long long rowbest[TS];
+  __shared__ int rowtok[TS];
+  const T *Kc = reinterpret_cast<const T *>(im.Kc);
+  const T *Kcen = reinterpret_cast<const T *>(im.Kcen);
+  const auto *rnt = rn_tok<D>(im);
+  const auto *rnc = rn_cen<D>(im);
+  for (int tile = blockIdx.x; tile < ntm * ntn; tile += gridDim.x) {
+    const int tm = tile / ntn, tn = tile % ntn;
+    if (t < TS) {
+      rowbest[t] = kBestInit;
+      const int g = tm * TS + t;
+      rowtok[t] = g < nrows ? (mode == ROWS_ALL ? g : list[g]) : -1;
+    }
+    __syncthreads();
+    acc_t acc[4][4];
+    tile_dots<T, acc_t>(
+        [&](int r) { const int tok = rowtok[r]; return tok >= 0 ? Kc + (size_t)tok * im.ldKc : (const T *)nullptr; },
+        [&](int r) { const int g = tn * TS + r; return g < C ? Kcen + (size_t)g * bt.d_k : (const T *)nullptr; },
+        bt.d_k, As, Bs, acc);
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+      const int tok = rowtok[ty * 4 + a];
+      if (tok < 0) continue;
+      const auto rni = rnt[tok];
+      unsigned long long bestv = kBestInit;
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        const int c = tn * TS + tx * 4 + b;
+        if (c >= C) continue;
+        const float dd = (float)D::dist(acc[a][b], rni, rnc[c]);
+        const unsigned long long pk = ((unsigned long long)__float_as_uint(dd) << 32) | (unsigned)c;
+        bestv = pk < bestv ? pk : bestv;
+      }
+      atomicMin(&rowbest[ty * 4 + a], bestv);
+    }
+    __syncthreads();
+    if (t < TS && rowtok[t] >= 0) atomicMin(&im.best[rowtok[t]], rowbest[t]);
+    __syncthreads();
+  }
+}
+
+// ---- labels -----------------------------------------------------------------------------------
+// survivors: cluster id of the nearest centre (a centre: its own id); pruned tokens: that id iff
+// the distance is strictly below alpha * d_c, else -1.
+template <typename T>
+__global__ void __launch_bounds__(256) k_label(const __grid_constant__ Batch bt, int mode) {
+  using D = typename DistOf<T>::type;
+  const ImgDesc &im = bt.img[blockIdx.y];
+  const int nrows = mode == ROWS_ALL ? im.N : (mode == ROWS_KEPT_LIST ? *im.q_ptr : *im.m_ptr);
+  int joined = 0, dropped = 0, band = 0;
+  for (int g = blockIdx.x * 256 + threadIdx.x; g < nrows; g += gridDim.x * 256) {
+    int tok, r;                                   // r >= 0: survivor position; < 0: pruned
+    if (mode == ROWS_ALL) { tok = g; r = im.slot[g]; }
+    else if (mode == ROWS_KEPT_LIST) { tok = im.kept_idx[g]; r = g; }
+    else { tok = im.pruned_idx[g]; r = -1; }
+    const unsigned long long pk = im.best[tok];
+    int lab = (int)(pk & 0xFFFFFFFFull);
+    const float dd = __uint_as_float((uint32_t)(pk >> 32));
+    if (r >= 0) {
+      if ((im.cmask[r >> 5] >> (r & 31)) & 1u) lab = im.cid[r];
+    } else {
+      if (D::in_band_t(dd, im)) ++band;
+      if (D::below_t(dd, im)) ++joined; else { lab = -1; ++dropped; }
+    }
+    im.label[tok] = lab;
+    if (im.label_user) im.label_user[tok] = lab;
+  }
+  // warp-aggregated counters
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    joined += __shfl_xor_sync(0xffffffffu, joined, o);
+    dropped += __shfl_xor_sync(0xffffffffu, dropped, o);
+    band += __shfl_xor_sync(0xffffffffu, band, o);
+  }
+  if ((threadIdx.x & 31) == 0) {
+    if (joined) { atomicAdd(&im.cnt[PACT_CNT_R], joined); }
+    if (dropped) atomicAdd(&im.cnt[PACT_CNT_DISCARDED], dropped);
+    if (band) atomicAdd(&im.cnt[PACT_CNT_BAND_ADC], band);
+  }
+}
+
+// ---- launchers ---------------------------------------------------------------------------------
+
+cudaError_t cluster_configure(ClusterCfg *cfg) {
+  int dev = 0, sms = 0, per_sm = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return e;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_centers, 256, 0);
+  if (e != cudaSuccess) return e;
+  cfg->sm_count = sms;
+  cfg->centers_grid = sms * (per_sm < 1 ? 1 : (per_sm > 4 ? 4 : per_sm));
+  return cudaSuccess;
+}
+
+#define PACT_DISPATCH(bf16, KERNEL, ...)                       \
+  do {                                                         \
+    if (bf16) KERNEL<__nv_bfloat16> __VA_ARGS__;               \
+    else KERNEL<float> __VA_ARGS__;                            \
+  } while (0)
+
+void launch_keynorm_gather(const Batch &bt, int maxN, bool bf16, bool all_tokens, cudaStream_t st) {
+  dim3 grid((maxN + 7) / 8, bt.B);
+  PACT_DISPATCH(bf16, k_keynorm_gather, <<<grid, 256, 0, st>>>(bt, all_tokens ? 1 : 0));
+}
+
+void launch_center_key_gather(const Batch &bt, int maxN, bool bf16, cudaStream_t st) {
+  dim3 grid((maxN + 7) / 8, bt.B);
+  PACT_DISPATCH(bf16, k_center_key_gather, <<<grid, 256, 0, st>>>(bt));
+}
+
+static int tile_grid(long long tiles, int cap) { return (int)(tiles < 1 ? 1 : (tiles > cap ? cap : tiles)); }
+
+void launch_gram(const Batch &bt, int maxN, bool bf16, const ClusterCfg &cfg, cudaStream_t st) {
+  const long long nt = (maxN + TS - 1) / TS;
+  dim3 grid(tile_grid(nt * nt, cfg.sm_count * 8), bt.B);
+  PACT_DISPATCH(bf16, k_gram_simt, <<<grid, 256, 0, st>>>(bt));
+}
+
+void launch_rank(const Batch &bt, int maxN, const ClusterCfg &cfg, cudaStream_t st) {
+  const long long nb = (maxN + 255) / 256;
+  dim3 grid(tile_grid(nb * nb, cfg.sm_count * 8), bt.B);
+  k_rank<<<grid, 256, 0, st>>>(bt);
+}
+
+cudaError_t launch_centers(const Batch &bt, const ClusterCfg &cfg, cudaStream_t st) {
+  void *args[] = {(void *)&bt};
+  return cudaLaunchCooperativeKernel((const void *)k_centers, dim3(cfg.centers_grid), dim3(256), args, 0, st);
+}
+
+void launch_centers_finalize(const Batch &bt, int maxN, bool bf16, const ClusterCfg &cfg, cudaStream_t st) {
+  int maxWp = 0;
+  for (int b = 0; b < bt.B; ++b) maxWp = bt.img[b].Wp > maxWp ? bt.img[b].Wp : maxWp;
+  dim3 grid(tile_grid((maxN + 7) / 8, cfg.sm_count * 2), bt.B);
+  const size_t sm = (size_t)(maxWp + 1) * sizeof(int);
+  PACT_DISPATCH(bf16, k_centers_finalize, <<<grid, 256, sm, st>>>(bt));
+}
+
+void launch_assign(const Batch &bt, int maxN, bool bf16, RowMode mode, const ClusterCfg &cfg, cudaStream_t st) {
+  const long long nt = (maxN + TS - 1) / TS;
+  dim3 grid(tile_grid(nt * nt, cfg.sm_count * 8), bt.B);
+  PACT_DISPATCH(bf16, k_assign_simt, <<<grid, 256, 0, st>>>(bt, (int)mode));
+}
+
+void launch_label(const Batch &bt, int maxN, bool bf16, RowMode mode, cudaStream_t st) {
+  dim3 grid(tile_grid((maxN + 255) / 256, 1 << 16), bt.B);
+  PACT_DISPATCH(bf16, k_label, <<<grid, 256, 0, st>>>(bt, (int)mode));
+}
+
+}  // namespace pact

@@ -1,0 +1,173 @@
+// Shared device-side declarations of the PACT reduction library (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/pact.h"
+
+namespace pact {
+
+constexpr int kMaxBatchPerLaunch = 16;   // images described by one kernel parameter block
+constexpr int kRowsPerCta = 32;          // visual tokens handled by one CTA of the EUTI kernels
+constexpr uint32_t kRhoShift = 30;       // density terms are summed as integers scaled by 2^30
+constexpr unsigned long long kBestInit = 0xFFFFFFFFFFFFFFFFull;
+constexpr int kSpinLimit = 1 << 20;      // passes a centre-selection warp makes before it gives up
+
+// Per-image device pointers: the caller's buffers and the slices of the workspace.
+struct ImgDesc {
+  // caller
+  const void *H, *Ke, *Q, *Kc;
+  long long ldH, ldKe, ldQ, ldKc, ldHo;
+  const int32_t *P;
+  void *H_out;
+  int32_t *P_out, *size_out, *label_user, *counters_user;
+  float *score_user;
+  unsigned char *keep_user;
+  int n_total, vis_start, N;
+  // parameters
+  int m_target;          // number of tokens the percentile aims to prune
+  float d_c, inv_dn_log2e, t_reinc;
+  double d_c64, inv_dn64, t_reinc64;
+  unsigned flags;
+  // workspace
+  double *qpart;         // [G][n_qcols] partial column sums of Q
+  double *qg;            // [n_qcols] global query
+  double *E;             // [N][n_qh] exp(logit - CTA max)
+  double *part;          // [G][n_qh][2] per-CTA (max, sum)
+  double *fac;           // [G][n_qh] exp(CTA max - max) / (Z n_qh)
+  double *nrm;           // [N] hidden-state norms
+  float *score;          // [N]
+  unsigned char *keep;   // [N]
+  int32_t *slot;         // [N] position in kept list, or -1-position in pruned list
+  int32_t *kept_idx;     // [N]
+  int32_t *pruned_idx;   // [N]
+  float *rn;             // [N] 1/|k_i| of the clustering keys, token order
+  double *rn64;          // [N] same in double (fp32-input path)
+  void *Kp;              // [Np][d_k] gathered keys of the survivors
+  float *rnk;            // [Np] 1/|k| in survivor order
+  double *rnk64;         // [Np]
+  unsigned long long *rho_fix;  // [Np] integer density
+  float *rho;            // [Np]
+  uint32_t *adj;         // [Np][Wp] adjacency bits (d <= d_c), later masked to earlier neighbours
+  int32_t *rank;         // [Np]
+  uint32_t *cmask;       // [Wp] centres
+  uint32_t *rmask;       // [Wp] removed (within d_c of an earlier centre)
+  void *Kcen;            // [Np][d_k] centre keys in cluster-id order
+  float *rnc;            // [Np]
+  double *rnc64;         // [Np]
+  int32_t *center_idx;   // [Np] token index of centre c
+  int32_t *cid;          // [Np] cluster id of survivor r if it is a centre
+  unsigned long long *best;  // [N] packed (distance bits << 32 | cluster id)
+  int32_t *label;        // [N]
+  int32_t *cnt;          // [PACT_N_COUNTERS] + scratch: [16] qsum ticket, [17] logit ticket
+  const int32_t *q_ptr;  // where the number of survivors lives (cnt[Q] or the caller's q_dev)
+  const int32_t *m_ptr;  // where the number of pruned tokens lives
+  const int32_t *C_ptr;  // where the number of clusters lives
+  const int32_t *cidx_ptr;  // token index of centre c (workspace or caller)
+  float *rho_user;       // optional outputs of the stage calls
+  int32_t *center_idx_user, *C_user, *r_user;
+  int Np, Wp;            // padded survivor capacity and words per adjacency row
+};
+
+struct Batch {
+  ImgDesc img[kMaxBatchPerLaunch];
+  int B;
+  int d, n_qh, n_kvh, d_h, d_k, n_qcols;
+};
+
+// ---- element access ----------------------------------------------------------------------
+
+template <typename T> struct Vec;      // 16-byte vector of T
+template <> struct Vec<__nv_bfloat16> { static constexpr int N = 8; };
+template <> struct Vec<float> { static constexpr int N = 4; };
+
+// Loads 16 bytes and widens to float.
+template <typename T> __device__ __forceinline__ void load_vec(const T *p, float (&out)[Vec<T>::N]);
+
+template <> __device__ __forceinline__ void load_vec<__nv_bfloat16>(const __nv_bfloat16 *p, float (&out)[8]) {
+  uint4 v = *reinterpret_cast<const uint4 *>(p);
+  uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    out[2 * i] = __uint_as_float(w[i] << 16);
+    out[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+  }
+}
+template <> __device__ __forceinline__ void load_vec<float>(const float *p, float (&out)[4]) {
+  float4 v = *reinterpret_cast<const float4 *>(p);
+  out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
+}
+
+__device__ __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ float to_float(float v) { return v; }
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Sum of squares of one row: each 16-byte vector is summed in float (the squares of bf16
+// values are exact in float), the vectors are accumulated in double.
+template <typename T>
+__device__ __forceinline__ double row_sumsq(const T *row, int n, int lane) {
+  constexpr int V = Vec<T>::N;
+  double acc = 0.0;
+  for (int v = lane; v * V < n; v += 32) {
+    float x[V];
+    load_vec<T>(row + (size_t)v * V, x);
+    if (sizeof(T) == 2) {
+      float s = 0.f;
+#pragma unroll
+      for (int i = 0; i < V; ++i) s = fmaf(x[i], x[i], s);
+      acc += (double)s;
+    } else {
+#pragma unroll
+      for (int i = 0; i < V; ++i) acc = fma((double)x[i], (double)x[i], acc);
+    }
+  }
+  return warp_sum(acc);
+}
+
+// ---- distance epilogue: the one place that turns a dot product into a distance ------------
+
+struct DistF {   // bf16 inputs: float arithmetic
+  using acc_t = float;
+  using rn_t = float;
+  __device__ static __forceinline__ float dist(float dot, float rn_i, float rn_j) {
+    float c = (dot * rn_i) * rn_j;
+    return fminf(fmaxf(1.0f - c, 0.0f), 2.0f);
+  }
+  __device__ static __forceinline__ uint32_t term(float d, const ImgDesc &im) {
+    float e = exp2f(-d * im.inv_dn_log2e);
+    return __float2uint_rn(e * (float)(1u << kRhoShift));
+  }
+  __device__ static __forceinline__ bool within(float d, const ImgDesc &im) { return d <= im.d_c; }
+  __device__ static __forceinline__ bool in_band(float d, const ImgDesc &im) { return fabsf(d - im.d_c) <= 1e-6f; }
+  __device__ static __forceinline__ bool below_t(float d, const ImgDesc &im) { return d < im.t_reinc; }
+  __device__ static __forceinline__ bool in_band_t(float d, const ImgDesc &im) { return fabsf(d - im.t_reinc) <= 1e-6f; }
+};
+
+struct DistD {   // fp32 inputs: double arithmetic
+  using acc_t = double;
+  using rn_t = double;
+  __device__ static __forceinline__ double dist(double dot, double rn_i, double rn_j) {
+    double c = (dot * rn_i) * rn_j;
+    return fmin(fmax(1.0 - c, 0.0), 2.0);
+  }
+  __device__ static __forceinline__ uint32_t term(double d, const ImgDesc &im) {
+    double e = exp(-d * im.inv_dn64);
+    return (uint32_t)__double2uint_rn(e * (double)(1u << kRhoShift));
+  }
+  __device__ static __forceinline__ bool within(double d, const ImgDesc &im) { return d <= im.d_c64; }
+  __device__ static __forceinline__ bool in_band(double d, const ImgDesc &im) { return fabs(d - im.d_c64) <= 1e-6; }
+  __device__ static __forceinline__ bool below_t(double d, const ImgDesc &im) { return d < im.t_reinc64; }
+  __device__ static __forceinline__ bool in_band_t(double d, const ImgDesc &im) { return fabs(d - im.t_reinc64) <= 1e-6; }
+};
+
+template <typename T> struct DistOf;
+template <> struct DistOf<__nv_bfloat16> { using type = DistF; };
+template <> struct DistOf<float> { using type = DistD; };
+
+}  // namespace pact

@@ -1,0 +1,37 @@
+// Launchers of the PACT kernels (host side); one translation unit per stage group.
+#pragma once
+#include "common.cuh"
+
+namespace pact {
+
+constexpr int kMergeMaxD = 256 * 4 * 8;   // widest hidden state the merge kernel holds in registers
+
+// how a kernel finds its rows
+enum RowMode { ROWS_ALL = 0, ROWS_KEPT_LIST = 1, ROWS_PRUNED_LIST = 2 };
+
+// euti.cu
+void launch_qsum(const Batch &bt, int maxN, bool bf16, cudaStream_t st);
+void launch_logit_norm(const Batch &bt, int maxN, bool bf16, cudaStream_t st);
+void launch_score_select(const Batch &bt, bool score, bool select, cudaStream_t st);
+cudaError_t euti_configure(int n_qcols, int n_qh);
+
+// cluster.cu
+struct ClusterCfg {
+  int sm_count;
+  int centers_grid;     // CTAs of the cooperative centre-selection kernel
+};
+cudaError_t cluster_configure(ClusterCfg *cfg);
+// gathers survivor keys and inverse norms; all_tokens: also every token's inverse norm
+void launch_keynorm_gather(const Batch &bt, int maxN, bool bf16, bool all_tokens, cudaStream_t st);
+void launch_center_key_gather(const Batch &bt, int maxN, bool bf16, cudaStream_t st);
+void launch_gram(const Batch &bt, int maxN, bool bf16, const ClusterCfg &cfg, cudaStream_t st);
+void launch_rank(const Batch &bt, int maxN, const ClusterCfg &cfg, cudaStream_t st);
+cudaError_t launch_centers(const Batch &bt, const ClusterCfg &cfg, cudaStream_t st);
+void launch_centers_finalize(const Batch &bt, int maxN, bool bf16, const ClusterCfg &cfg, cudaStream_t st);
+void launch_assign(const Batch &bt, int maxN, bool bf16, RowMode mode, const ClusterCfg &cfg, cudaStream_t st);
+void launch_label(const Batch &bt, int maxN, bool bf16, RowMode mode, cudaStream_t st);
+
+// merge.cu
+void launch_merge(const Batch &bt, bool in_bf16, bool out_bf16, const ClusterCfg &cfg, cudaStream_t st);
+
+}  // namespace pact

