@@ -16,6 +16,7 @@ struct pact_ctx {
   pact_dtype in, out;
   int elt;                 // bytes per input element
   ClusterCfg ccfg;
+  bool umma;               // bf16 keys of a width the tcgen05 tile kernels take
   int device;
   char err[256];
   long long launches;      // kernels launched by this context so far
@@ -217,12 +218,14 @@ pact_status pact_create(pact_ctx **out, int d, int n_qh, int n_kvh, int d_h, pac
   }
   if (e == cudaSuccess) e = euti_configure(c->n_qcols, c->n_qh);
   if (e == cudaSuccess) e = cluster_configure(&c->ccfg);
+  if (e == cudaSuccess && in == PACT_BF16) e = umma_configure();
   if (e != cudaSuccess) {
     pact_status s = fail_cuda(ctx, e, "pact_create");
     (void)s;
     delete c;
     return PACT_ERR_CUDA;
   }
+  c->umma = in == PACT_BF16 && umma_supported(c->d_k);
   *out = c;
   return PACT_OK;
 }
@@ -346,11 +349,13 @@ pact_status pact_dbdpc(pact_ctx *ctx, const void *K, int64_t ldK, int N, const i
   m.rho_user = rho; m.center_idx_user = center_idx; m.C_user = C_dev; m.label_user = label;
   CK(cudaMemsetAsync(m.cnt, 0, 32 * sizeof(int32_t), st));
   launch_keynorm_gather(bt, N, bf, false, st);
-  launch_gram(bt, N, bf, ctx->ccfg, st);
+  if (ctx->umma) CK(launch_gram_umma(bt, N, ctx->ccfg, st));
+  else launch_gram(bt, N, bf, ctx->ccfg, st);
   launch_rank(bt, N, ctx->ccfg, st);
   CK(launch_centers(bt, ctx->ccfg, st));
   launch_centers_finalize(bt, N, bf, ctx->ccfg, st);
-  launch_assign(bt, N, bf, ROWS_KEPT_LIST, ctx->ccfg, st);
+  if (ctx->umma) CK(launch_assign_umma(bt, N, true, ctx->ccfg, st));
+  else launch_assign(bt, N, bf, ROWS_KEPT_LIST, ctx->ccfg, st);
   launch_label(bt, N, bf, ROWS_KEPT_LIST, st);
   ctx->launches += 7;
   CK(cudaGetLastError());
@@ -468,11 +473,15 @@ pact_status pact_reduce(pact_ctx *ctx, const pact_image *imgs, int B, const pact
     launch_logit_norm(bt, cmaxN, bf, st);           CK(mark());
     launch_score_select(bt, true, true, st);        CK(mark());
     launch_keynorm_gather(bt, cmaxN, bf, true, st); CK(mark());
-    launch_gram(bt, cmaxN, bf, ctx->ccfg, st);      CK(mark());
+    if (ctx->umma) CK(launch_gram_umma(bt, cmaxN, ctx->ccfg, st));
+    else launch_gram(bt, cmaxN, bf, ctx->ccfg, st);
+    CK(mark());
     launch_rank(bt, cmaxN, ctx->ccfg, st);          CK(mark());
     CK(launch_centers(bt, ctx->ccfg, st));          CK(mark());
     launch_centers_finalize(bt, cmaxN, bf, ctx->ccfg, st);  CK(mark());
-    launch_assign(bt, cmaxN, bf, ROWS_ALL, ctx->ccfg, st);  CK(mark());
+    if (ctx->umma) CK(launch_assign_umma(bt, cmaxN, false, ctx->ccfg, st));
+    else launch_assign(bt, cmaxN, bf, ROWS_ALL, ctx->ccfg, st);
+    CK(mark());
     launch_label(bt, cmaxN, bf, ROWS_ALL, st);      CK(mark());
     launch_merge(bt, bf, ctx->out == PACT_BF16, ctx->ccfg, st);  CK(mark());
     ctx->launches += 11;

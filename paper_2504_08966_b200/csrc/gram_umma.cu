@@ -1,0 +1,368 @@
+// tcgen05 tile kernels for bf16 keys (sm_100a): the all-pairs distance pass of DBDPC (Eq. 5) with
+// the density (Eq. 6) and the d <= d_c adjacency fused into the epilogue, and the rows x centres
+// nearest-centre pass (Algorithm 2 assignment, Eq. 8).  Nothing of the distance matrix reaches
+// memory: accumulators live in tensor memory and are consumed from there.
+//
+// One persistent CTA per SM, 192 threads:
+//   warp 0      TMA producer: 128-byte-swizzled K-slabs of the two operands into a shared-memory ring
+//   warp 1      allocates tensor memory, issues tcgen05.mma (128 x BN x 16, bf16 -> fp32)
+//   warps 2-5   epilogue: tcgen05.ld of their 32-lane quadrant, distance arithmetic of common.cuh
+// Two accumulators (2 x BN columns of tensor memory) let the epilogue of tile t overlap the MMAs of
+// tile t+1.  Every mbarrier wait is bounded; when one runs out the CTA raises the image's status
+// word, drains what it armed, frees its tensor memory and returns.
+#include <cuda.h>
+
+#include "kernels.cuh"
+
+namespace pact {
+
+namespace {
+
+constexpr int BM = 128;           // rows per tile (UMMA M)
+constexpr int BN = 256;           // columns per tile (UMMA N)
+constexpr int BK = 64;            // bf16 elements per K-slab = one 128-byte swizzle row
+constexpr int STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2;
+constexpr int B_BYTES = BN * BK * 2;
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int TMEM_COLS = 2 * BN; // 512: all of an SM's tensor memory
+constexpr unsigned long long kWaitNs = 1000000000ull;   // one second per wait, then give up
+
+struct TmapSet {
+  CUtensorMap a[kMaxBatchPerLaunch];
+  CUtensorMap b[kMaxBatchPerLaunch];
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait: false when kWaitNs of wall time have passed without the phase completing.
+__device__ __noinline__ bool mbar_wait_slow(uint64_t *bar, uint32_t parity) {
+  const unsigned long long t0 = global_ns();
+  for (uint32_t i = 0;; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 255u) == 255u && global_ns() - t0 > kWaitNs) return false;
+  }
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
+  for (int i = 0; i < 64; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity);
+}
+
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, uint64_t *bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t *slot, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accum) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t *bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory operand descriptor: K-major rows of 128 bytes, 128-byte swizzle, 8-row groups
+// 1024 bytes apart, descriptor version 1.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// kind::f16 instruction descriptor: fp32 accumulate, bf16 x bf16, both operands K-major.
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+struct Shared {
+  uint64_t full[STAGES], empty[STAGES], acc_full[2], acc_empty[2];
+  uint32_t tmem_base;
+  int abort;
+  float rn_col[4][BN];          // one copy per epilogue warp
+};
+
+enum { MODE_GRAM = 0, MODE_ASSIGN = 1 };
+
+}  // namespace
+
+// grid (X, B), 192 threads, dynamic smem = 1024 (alignment slack) + STAGES * STAGE_BYTES.
+// kept_rows (assignment only): rows are the gathered survivors (Kp, rnk) instead of all tokens.
+template <int MODE>
+__global__ void __launch_bounds__(192, 1) k_tiles_umma(const __grid_constant__ Batch bt,
+                                                       const __grid_constant__ TmapSet tm, int kept_rows) {
+  const ImgDesc &im = bt.img[blockIdx.y];
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ Shared sh;
+  uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  int nrows, ncols;
+  if (MODE == MODE_GRAM) { nrows = *im.q_ptr; ncols = nrows; }
+  else { nrows = kept_rows ? *im.q_ptr : im.N; ncols = *im.C_ptr; }
+  const int ntm = (nrows + BM - 1) / BM, ntn = (ncols + BN - 1) / BN;
+  const int ntiles = ntm * ntn;
+  if ((int)blockIdx.x >= ntiles) return;            // uniform: nothing allocated yet
+  const int nslab = bt.d_k / BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&sh.acc_full[a], 1); mbar_init(&sh.acc_empty[a], 4); }
+    sh.abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(&sh.tmem_base, TMEM_COLS);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = sh.tmem_base;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      const CUtensorMap *ma = &tm.a[blockIdx.y], *mb = &tm.b[blockIdx.y];
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < ntiles; tile += gridDim.x) {
+        const int tmi = tile / ntn, tni = tile % ntn;
+        for (int ks = 0; ks < nslab; ++ks, ++it) {
+          const int s = it % STAGES;
+          if (!mbar_wait(&sh.empty[s], ((it / STAGES) & 1) ^ 1)) { ok = false; break; }
+          uint8_t *a_dst = ring + (size_t)s * STAGE_BYTES, *b_dst = a_dst + A_BYTES;
+          mbar_arrive_expect_tx(&sh.full[s], STAGE_BYTES);
+          tma_load_2d(a_dst, ma, &sh.full[s], ks * BK, tmi * BM);
+          tma_load_2d(b_dst, mb, &sh.full[s], ks * BK, tni * BN);
+          tma_load_2d(b_dst + B_BYTES / 2, mb, &sh.full[s], ks * BK, tni * BN + BN / 2);
+        }
+      }
+      if (!ok) atomicExch(&sh.abort, 1);
+      // drain: every armed stage completes before the CTA may exit (its copies target this smem)
+      const uint32_t armed = it < (uint32_t)STAGES ? it : (uint32_t)STAGES;
+      for (uint32_t k = 0; k < armed; ++k) {
+        const uint32_t j = it - 1 - k;
+        mbar_wait(&sh.full[j % STAGES], (j / STAGES) & 1);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      uint32_t it = 0, tcount = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < ntiles; tile += gridDim.x, ++tcount) {
+        const uint32_t a = tcount & 1;
+        if (!mbar_wait(&sh.acc_empty[a], ((tcount >> 1) & 1) ^ 1)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + a * BN;
+        for (int ks = 0; ks < nslab; ++ks, ++it) {
+          const int s = it % STAGES;
+          if (!mbar_wait(&sh.full[s], (it / STAGES) & 1)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_addr = smem_u32(ring + (size_t)s * STAGE_BYTES), b_addr = a_addr + A_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k)
+            umma_bf16(d_tmem, smem_desc(a_addr + k * 32), smem_desc(b_addr + k * 32), kIdesc, (ks | k) != 0);
+          umma_commit(&sh.empty[s]);               // frees the slab once these MMAs have read it
+        }
+        if (ok) umma_commit(&sh.acc_full[a]);      // accumulator complete
+      }
+      if (!ok) atomicExch(&sh.abort, 1);
+    }
+  } else {
+    // ---------------- epilogue ----------------
+    const int qd = warp & 3;                        // tensor-memory lane quadrant of this warp
+    float *rn_col = sh.rn_col[qd];
+    uint32_t tcount = 0;
+    int band = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; ok && tile < ntiles; tile += gridDim.x, ++tcount) {
+      const int tmi = tile / ntn, tni = tile % ntn;
+      const uint32_t a = tcount & 1;
+      // inverse norms of this tile's columns
+      __syncwarp();
+      for (int c = lane; c < BN; c += 32) {
+        const int gj = tni * BN + c;
+        rn_col[c] = gj < ncols ? (MODE == MODE_GRAM ? im.rnk[gj] : im.rnc[gj]) : 0.f;
+      }
+      __syncwarp();
+      if (!__all_sync(0xffffffffu, mbar_wait(&sh.acc_full[a], (tcount >> 1) & 1))) { ok = false; break; }
+      tc_fence_after();
+      const int row = tmi * BM + qd * 32 + lane;
+      const bool row_ok = row < nrows;
+      const bool kept_space = MODE == MODE_GRAM || kept_rows;
+      const float rni = row_ok ? (kept_space ? im.rnk[row] : im.rn[row]) : 0.f;
+      const uint32_t taddr = tmem_base + a * BN + ((uint32_t)(qd * 32) << 16);
+      unsigned long long rowsum = 0ull;
+      unsigned long long best = kBestInit;
+#pragma unroll 1
+      for (int ch = 0; ch < BN / 32; ++ch) {
+        uint32_t v[32];
+        tmem_ld32(taddr + ch * 32, v);
+        tmem_ld_wait();
+        const int c0 = tni * BN + ch * 32;
+        if (c0 >= ncols) continue;                  // uniform
+        if (MODE == MODE_GRAM) {
+          uint32_t bits = 0u;
+          unsigned long long s = 0ull;
+#pragma unroll
+          for (int k = 0; k < 32; ++k) {
+            const int gj = c0 + k;
+            float dd = DistF::dist(__uint_as_float(v[k]), rni, rn_col[ch * 32 + k]);
+            if (gj == row) dd = 0.f;
+            if (gj < ncols) {
+              s += DistF::term(dd, im);
+              if (DistF::within(dd, im)) bits |= 1u << k;
+              if (row < gj && DistF::in_band(dd, im)) ++band;
+            }
+          }
+          if (row_ok) {
+            rowsum += s;
+            im.adj[(size_t)row * im.Wp + (c0 >> 5)] = bits;
+          }
+        } else {
+#pragma unroll
+          for (int k = 0; k < 32; ++k) {
+            const int gj = c0 + k;
+            const float dd = DistF::dist(__uint_as_float(v[k]), rni, rn_col[ch * 32 + k]);
+            const unsigned long long pk = ((unsigned long long)__float_as_uint(dd) << 32) | (unsigned)gj;
+            if (gj < ncols && pk < best) best = pk;
+          }
+        }
+      }
+      // the accumulator may be overwritten once all four epilogue warps have read it
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.acc_empty[a]);
+      if (row_ok) {
+        if (MODE == MODE_GRAM) atomicAdd(&im.rho_fix[row], rowsum);
+        else atomicMin(&im.best[kept_rows ? im.kept_idx[row] : row], best);
+      }
+    }
+    if (!ok) atomicExch(&sh.abort, 1);
+    if (MODE == MODE_GRAM && band) atomicAdd(&im.cnt[PACT_CNT_BAND_DC], band);
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 1) tmem_dealloc(tmem_base, TMEM_COLS);
+  if (threadIdx.x == 0 && sh.abort) atomicMin(&im.cnt[PACT_CNT_STATUS], (int)PACT_ERR_TIMEOUT);
+}
+
+// ---- host side -----------------------------------------------------------------------------------
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+bool encode_rows(CUtensorMap *map, const void *base, long long rows, long long ld_elems, int d_k) {
+  const cuuint64_t dims[2] = {(cuuint64_t)d_k, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)ld_elems * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)BM};
+  const cuuint32_t estr[2] = {1, 1};
+  return g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+constexpr size_t kUmmaSmem = 1024 + (size_t)STAGES * STAGE_BYTES;
+
+}  // namespace
+
+cudaError_t umma_configure() {
+  void *fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+  if (e != cudaSuccess) return e;
+  if (qres != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
+  g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  e = cudaFuncSetAttribute(k_tiles_umma<MODE_GRAM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kUmmaSmem);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(k_tiles_umma<MODE_ASSIGN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kUmmaSmem);
+}
+
+bool umma_supported(int d_k) { return g_encode != nullptr && d_k % BK == 0; }
+
+static int umma_grid_x(int max_rows, int max_cols, int B, int sms) {
+  const long long tiles = (long long)((max_rows + BM - 1) / BM) * ((max_cols + BN - 1) / BN);
+  long long x = (sms + B - 1) / B;
+  if (x < 1) x = 1;
+  if (x > tiles) x = tiles;
+  return (int)(x < 1 ? 1 : x);
+}
+
+cudaError_t launch_gram_umma(const Batch &bt, int maxN, const ClusterCfg &cfg, cudaStream_t st) {
+  TmapSet tm;
+  for (int b = 0; b < bt.B; ++b) {
+    const ImgDesc &im = bt.img[b];
+    if (!encode_rows(&tm.a[b], im.Kp, im.Np, bt.d_k, bt.d_k)) return cudaErrorInvalidValue;
+    tm.b[b] = tm.a[b];
+  }
+  dim3 grid(umma_grid_x(maxN, maxN, bt.B, cfg.sm_count), bt.B);
+  k_tiles_umma<MODE_GRAM><<<grid, 192, kUmmaSmem, st>>>(bt, tm, 0);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_assign_umma(const Batch &bt, int maxN, bool kept_rows, const ClusterCfg &cfg, cudaStream_t st) {
+  TmapSet tm;
+  for (int b = 0; b < bt.B; ++b) {
+    const ImgDesc &im = bt.img[b];
+    if (kept_rows) {
+      if (!encode_rows(&tm.a[b], im.Kp, im.Np, bt.d_k, bt.d_k)) return cudaErrorInvalidValue;
+    } else if (!encode_rows(&tm.a[b], im.Kc, im.N, im.ldKc, bt.d_k)) return cudaErrorInvalidValue;
+    if (!encode_rows(&tm.b[b], im.Kcen, im.Np, bt.d_k, bt.d_k)) return cudaErrorInvalidValue;
+  }
+  dim3 grid(umma_grid_x(maxN, maxN, bt.B, cfg.sm_count), bt.B);
+  k_tiles_umma<MODE_ASSIGN><<<grid, 192, kUmmaSmem, st>>>(bt, tm, kept_rows ? 1 : 0);
+  return cudaGetLastError();
+}
+
+}  // namespace pact

@@ -31,6 +31,12 @@ void launch_centers_finalize(const Batch &bt, int maxN, bool bf16, const Cluster
 void launch_assign(const Batch &bt, int maxN, bool bf16, RowMode mode, const ClusterCfg &cfg, cudaStream_t st);
 void launch_label(const Batch &bt, int maxN, bool bf16, RowMode mode, cudaStream_t st);
 
+// gram_umma.cu: tcgen05 versions of the two tile passes for bf16 keys whose width is a multiple of 64
+cudaError_t umma_configure();
+bool umma_supported(int d_k);
+cudaError_t launch_gram_umma(const Batch &bt, int maxN, const ClusterCfg &cfg, cudaStream_t st);
+cudaError_t launch_assign_umma(const Batch &bt, int maxN, bool kept_rows, const ClusterCfg &cfg, cudaStream_t st);
+
 // merge.cu
 void launch_merge(const Batch &bt, bool in_bf16, bool out_bf16, const ClusterCfg &cfg, cudaStream_t st);
 
