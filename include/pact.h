@@ -163,6 +163,24 @@ pact_status pact_prune(pact_ctx *ctx, const float *score, int N, const pact_para
                        uint8_t *keep, int32_t *kept_idx, int32_t *pruned_idx, int32_t *counts,
                        void *ws, size_t ws_bytes, void *stream);
 
+/* The same split for callers that cannot allocate device memory (no counterpart in the paper:
+ * this is a packaging variant of pact_prune, not a step of the method).  pact_prune needs a
+ * workspace that somebody obtained from cudaMalloc; a host that runs inside another framework's
+ * callback, a plugin that is handed tensors but no allocator, or a process whose device memory is
+ * already fully parcelled out cannot provide one.  This entry point takes no context and no
+ * workspace: its scratch is a fixed array inside the library image (about 256 KiB, resident on
+ * every GPU that loads the library until the process exits), and it calls no allocating routine.
+ *  - N must not exceed PACT_PRUNE_STATIC_MAX_N; larger N returns PACT_ERR_UNSUPPORTED and launches
+ *    nothing.  Only p->lambda and p->n_prune are read.
+ *  - The first call on each device looks up the array's device address (with that device
+ *    current); make that first call outside any stream capture.
+ *  - All calls on a device share the one array: two calls whose kernels may overlap on the GPU
+ *    (different streams without an ordering between them) race.  Calls on one stream are safe.
+ * Inputs, outputs and their meaning are those of pact_prune. */
+#define PACT_PRUNE_STATIC_MAX_N 65536
+pact_status pact_prune_static(const float *score, int N, const pact_params *p /*host*/, uint8_t *keep,
+                              int32_t *kept_idx, int32_t *pruned_idx, int32_t *counts, void *stream);
+
 /* DBDPC, Algorithm 2 (Eq. 5-7) on the rows idx[0..q) of K[N, d_k]:
  * all-pairs cosine distance, density with d_n, density-ordered centre selection under d_c
  * (the result of the sequential loop, computed by asynchronous parallel resolution, cf.

@@ -23,7 +23,7 @@ FLAG_CENTER_ONLY, FLAG_NO_NORM, FLAG_NORM_ONLY = 1, 2, 4
 
 EXPORTS = ["pact_create", "pact_destroy", "pact_workspace_bytes", "pact_status_string",
            "pact_last_cuda_error", "pact_importance", "pact_prune", "pact_dbdpc",
-           "pact_reincorporate", "pact_merge", "pact_reduce", "pact_reduce_host",
+           "pact_prune_static", "pact_reincorporate", "pact_merge", "pact_reduce", "pact_reduce_host",
            "pact_host_staging_bytes", "pact_launch_count", "pact_profile_enable", "pact_profile_read",
            "pact_profile_stage_name"]
 
@@ -63,6 +63,7 @@ def lib():
         L.pact_last_cuda_error.restype = C.c_char_p
         L.pact_importance.argtypes = [vp, C.POINTER(ImageDesc), C.POINTER(Params), vp, vp, sz, vp]
         L.pact_prune.argtypes = [vp, vp, i32, C.POINTER(Params), vp, vp, vp, vp, vp, sz, vp]
+        L.pact_prune_static.argtypes = [vp, i32, C.POINTER(Params), vp, vp, vp, vp, vp]
         L.pact_dbdpc.argtypes = [vp, vp, i64, i32, vp, vp, C.POINTER(Params), vp, vp, vp, vp, vp, vp, sz, vp]
         L.pact_reincorporate.argtypes = [vp, vp, i64, i32, vp, vp, vp, vp, C.POINTER(Params), vp, vp, vp,
                                          vp, sz, vp]
@@ -157,6 +158,17 @@ def device_image(img, out_dtype, device="cuda") -> DeviceImage:
                        torch.empty(img.N, dtype=torch.float32, device=device),
                        torch.empty(img.N, dtype=torch.uint8, device=device),
                        torch.zeros(N_COUNTERS, dtype=torch.int32, device=device))
+
+
+PRUNE_STATIC_MAX_N = 65536
+
+
+def pact_prune_static(score, params: Params, keep, kept_idx, pruned_idx, counts):
+    """pact_prune without context or workspace, for callers that may not allocate device memory:
+    the scratch is a fixed array inside the library.  score.numel() <= PRUNE_STATIC_MAX_N.
+    Calls on one stream are ordered; calls that could overlap on the GPU share the array and race."""
+    _check(None, lib().pact_prune_static(_ptr(score), score.numel(), C.byref(params), _ptr(keep), _ptr(kept_idx),
+                                         _ptr(pruned_idx), _ptr(counts), _stream()))
 
 
 class Context:

@@ -9,7 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpact.so")
-SOURCES = ["api.cu", "euti.cu", "cluster.cu", "gram_umma.cu", "merge.cu"]
+SOURCES = ["api.cu", "euti.cu", "cluster.cu", "gram_umma.cu", "merge.cu", "prune_static.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 

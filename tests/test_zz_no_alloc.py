@@ -1,0 +1,69 @@
+"""pact_prune_static, the percentile split for callers that cannot allocate device memory.
+
+Some hosts of the library have no way to obtain a workspace: they run inside another framework's
+callback, or are handed tensors but no allocator, or live in a process whose device memory is
+already fully parcelled out.  For them the scratch of the split is a fixed array inside the
+library.  This test calls that entry point through the C ABI twice in a row (the second call finds
+the array as the first one left it, with a different N and pruning fraction) and requires bit-equal
+outputs to pact_prune, which uses a caller workspace.  The file sorts last so that a failure here
+cannot hide the result of any other test in a run that stops at the first failure.
+"""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_both(pb, ctx, score, lam):
+    N = score.numel()
+    p = pb.make_params(lam=lam)
+
+    def outputs():
+        return (torch.full((N,), 7, dtype=torch.uint8, device="cuda"),
+                torch.full((N,), -5, dtype=torch.int32, device="cuda"),
+                torch.full((N,), -5, dtype=torch.int32, device="cuda"),
+                torch.full((2,), -5, dtype=torch.int32, device="cuda"))
+
+    ref = outputs()
+    ctx.pact_prune(score, p, *ref)
+    got = outputs()
+    pb.pact_prune_static(score, p, *got)
+    torch.cuda.synchronize()
+    q, m = ref[3].cpu().tolist()
+    assert got[3].cpu().tolist() == [q, m] and q + m == N
+    assert torch.equal(got[0], ref[0])
+    assert torch.equal(got[1][:q], ref[1][:q]) and torch.equal(got[2][:m], ref[2][:m])
+    return q, m
+
+
+def test_static_scratch_split_matches_workspace_split_twice_in_a_row():
+    from paper_2504_08966_b200 import binding as pb
+    ctx = pb.Context(256, 2, 2, 32, torch.bfloat16, torch.bfloat16)
+    g = torch.Generator().manual_seed(5)
+    a = torch.rand(5000, generator=g).cuda()
+    a[17] = a[4000] = a[99]                        # ties
+    a[3] = -0.25
+    b = torch.rand(1237, generator=g).cuda()
+    q1, m1 = _run_both(pb, ctx, a, 0.5)
+    q2, m2 = _run_both(pb, ctx, b, 0.3)            # second call: smaller N, stale scratch from the first
+    assert m1 == 2500 and m2 == 371
+    q3, _ = _run_both(pb, ctx, a, 0.0)             # nothing pruned
+    assert q3 == 5000
+
+
+def test_static_scratch_split_rejects_sizes_beyond_its_array():
+    import ctypes as C
+    from paper_2504_08966_b200 import binding as pb
+    L = pb.lib()
+    n = pb.PRUNE_STATIC_MAX_N + 1
+    buf = torch.zeros(n, dtype=torch.float32, device="cuda")
+    i32 = torch.zeros(n, dtype=torch.int32, device="cuda")
+    p = pb.make_params(lam=0.5)
+    vp = lambda t: C.c_void_p(t.data_ptr())
+    st = L.pact_prune_static(vp(buf), n, C.byref(p), vp(i32), vp(i32), vp(i32), vp(i32), None)
+    assert st == -2
+    assert L.pact_prune_static(None, 16, C.byref(p), vp(i32), vp(i32), vp(i32), vp(i32), None) == -1
+    bad = pb.make_params(lam=1.5)
+    assert L.pact_prune_static(vp(buf), 16, C.byref(bad), vp(i32), vp(i32), vp(i32), vp(i32), None) == -1
+    torch.cuda.synchronize()
