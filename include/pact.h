@@ -219,6 +219,21 @@ pact_status pact_reduce(pact_ctx *ctx, const pact_image *imgs /*host*/, int B,
                         const pact_params *params /*host*/, int params_stride, void *ws,
                         size_t ws_bytes, void *stream);
 
+/* ---- replayable form of pact_reduce (CUDA graph) --------------------------------------------- */
+
+/* Records the launch sequence of pact_reduce(ctx, imgs, B, params, params_stride, ws, ws_bytes) once
+ * into a CUDA graph; pact_graph_launch replays it on `stream` at a fraction of the launch cost (the
+ * path is a chain of short dependent kernels, so launch gaps matter).  The graph holds the pointers
+ * given here: the buffers and the workspace must stay valid and in place while it is used; their
+ * contents may change between launches.  One launch at a time per graph (they share the workspace).
+ * Nothing runs on the device during pact_graph_create. */
+typedef struct pact_graph pact_graph;
+pact_status pact_graph_create(pact_ctx *ctx, const pact_image *imgs /*host*/, int B,
+                              const pact_params *params /*host*/, int params_stride, void *ws,
+                              size_t ws_bytes, pact_graph **graph);
+pact_status pact_graph_launch(pact_graph *graph, void *stream);
+pact_status pact_graph_destroy(pact_graph *graph);
+
 /* Same computation with HOST buffers for one image: copies the inputs to the device, runs
  * pact_reduce, copies H_out/P_out/size_out/label/counters back and synchronises.
  * dev_in / dev_out are device staging buffers the caller provides (sizes from

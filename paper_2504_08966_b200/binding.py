@@ -25,7 +25,7 @@ EXPORTS = ["pact_create", "pact_destroy", "pact_workspace_bytes", "pact_status_s
            "pact_last_cuda_error", "pact_importance", "pact_prune", "pact_dbdpc",
            "pact_prune_static", "pact_reincorporate", "pact_merge", "pact_reduce", "pact_reduce_host",
            "pact_host_staging_bytes", "pact_launch_count", "pact_profile_enable", "pact_profile_read",
-           "pact_profile_stage_name"]
+           "pact_profile_stage_name", "pact_graph_create", "pact_graph_launch", "pact_graph_destroy"]
 
 
 class Params(C.Structure):
@@ -72,6 +72,9 @@ def lib():
         L.pact_reduce_host.argtypes = [vp, C.POINTER(ImageDesc), C.POINTER(Params), vp, sz, vp, sz, vp]
         L.pact_host_staging_bytes.argtypes = [vp, i32, i32]
         L.pact_host_staging_bytes.restype = sz
+        L.pact_graph_create.argtypes = [vp, C.POINTER(ImageDesc), i32, C.POINTER(Params), i32, vp, sz, C.POINTER(vp)]
+        L.pact_graph_launch.argtypes = [vp, vp]
+        L.pact_graph_destroy.argtypes = [vp]
         L.pact_launch_count.argtypes = [vp]
         L.pact_launch_count.restype = C.c_longlong
         L.pact_profile_enable.argtypes = [vp, i32]
@@ -158,6 +161,28 @@ def device_image(img, out_dtype, device="cuda") -> DeviceImage:
                        torch.empty(img.N, dtype=torch.float32, device=device),
                        torch.empty(img.N, dtype=torch.uint8, device=device),
                        torch.zeros(N_COUNTERS, dtype=torch.int32, device=device))
+
+
+class Graph:
+    """A recorded pact_reduce; launch() replays it on the current stream.  Keeps the tensors it
+    points at alive."""
+
+    def __init__(self, ctx, handle, images, ws):
+        self._ctx, self.handle, self._images, self._ws = ctx, handle, images, ws
+
+    def launch(self):
+        _check(self._ctx.handle, self._ctx._L.pact_graph_launch(self.handle, _stream()))
+
+    def close(self):
+        if self.handle:
+            self._ctx._L.pact_graph_destroy(self.handle)
+            self.handle = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 PRUNE_STATIC_MAX_N = 65536
@@ -256,6 +281,20 @@ class Context:
             parr, stride = (Params * B)(*params), 1
         w, n = self._ws()
         _check(self.handle, self._L.pact_reduce(self.handle, arr, B, parr, stride, w, n, _stream()))
+
+    def pact_graph_create(self, images, params):
+        """Records pact_reduce(images, params) as a replayable graph (see Graph)."""
+        B = len(images)
+        self.ensure_workspace(B, max(im.N for im in images))
+        arr = (ImageDesc * B)(*[im.desc() for im in images])
+        if isinstance(params, Params):
+            parr, stride = (Params * 1)(params), 0
+        else:
+            parr, stride = (Params * B)(*params), 1
+        w, n = self._ws()
+        h = C.c_void_p()
+        _check(self.handle, self._L.pact_graph_create(self.handle, arr, B, parr, stride, w, n, C.byref(h)))
+        return Graph(self, h, images, self.ws)
 
     def launch_count(self) -> int:
         return int(self._L.pact_launch_count(self.handle))

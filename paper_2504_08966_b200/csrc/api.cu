@@ -9,7 +9,7 @@
 
 using namespace pact;
 
-constexpr int kProfStages = 11;
+constexpr int kProfStages = 12;
 
 struct pact_ctx {
   int d, n_qh, n_kvh, d_h, d_k, n_qcols;
@@ -25,9 +25,15 @@ struct pact_ctx {
   cudaEvent_t ev[kProfStages + 1];
 };
 
+struct pact_graph {
+  pact_ctx *ctx;
+  cudaGraphExec_t exec;
+  int kernels;             // kernels one replay launches
+};
+
 static const char *const kStageNames[kProfStages] = {
-    "qsum", "logit_norm", "score_select", "keynorm_gather", "gram_density", "rank",
-    "centers", "centers_finalize", "assign", "label", "merge"};
+    "prepass", "logits", "scores", "select_gather", "gram_density", "rank",
+    "centers", "centers_finalize", "assign", "label", "lists", "merge"};
 
 namespace {
 
@@ -54,11 +60,10 @@ size_t carve_image(const pact_ctx *c, int N, char *base, ImgDesc *im) {
   m.Np = Np;
   m.Wp = Wp;
   cv.take(m.cnt, 32 * sizeof(int32_t));
-  cv.take(m.qpart, (size_t)G * c->n_qcols * sizeof(double));
+  cv.take(m.qpart, (size_t)kQPartRows * c->n_qcols * sizeof(double));
   cv.take(m.qg, (size_t)c->n_qcols * sizeof(double));
   cv.take(m.E, (size_t)N * c->n_qh * sizeof(double));
   cv.take(m.part, (size_t)G * c->n_qh * 2 * sizeof(double));
-  cv.take(m.fac, (size_t)G * c->n_qh * sizeof(double));
   cv.take(m.nrm, (size_t)N * sizeof(double));
   cv.take(m.score, (size_t)N * sizeof(float));
   cv.take(m.keep, (size_t)N);
@@ -83,6 +88,14 @@ size_t carve_image(const pact_ctx *c, int N, char *base, ImgDesc *im) {
   cv.take(m.cid, (size_t)Np * sizeof(int32_t));
   cv.take(m.best, (size_t)N * sizeof(unsigned long long));
   cv.take(m.label, (size_t)N * sizeof(int32_t));
+  const size_t nblk = ((size_t)N + 255) / 256;
+  m.bstride = Np + 8;
+  cv.take(m.blocklist, nblk * 256 * sizeof(int32_t));
+  cv.take(m.bstart, nblk * (size_t)m.bstride * sizeof(uint16_t));
+  cv.take(m.csize, (size_t)Np * sizeof(int32_t));
+  cv.take(m.cbase, (size_t)Np * sizeof(int32_t));
+  cv.take(m.cticket, (size_t)Np * sizeof(int32_t));
+  cv.take(m.mpart, ((size_t)N / 8 + 2) * c->d * sizeof(float));
   return cv.off;
 }
 
@@ -284,13 +297,14 @@ pact_status pact_importance(pact_ctx *ctx, const pact_image *img, const pact_par
   ImgDesc &m = bt.img[0];
   carve_image(ctx, img->N, (char *)ws, &m);
   fill_user(m, img);
+  m.Kc = nullptr;                        // no clustering keys in this stage
   m.score_user = score;
   set_params(m, p, img->N);
   point_counts_at_workspace(m);
   CK(cudaMemsetAsync(m.cnt, 0, 32 * sizeof(int32_t), st));
-  launch_qsum(bt, img->N, ctx->in == PACT_BF16, st);
-  launch_logit_norm(bt, img->N, ctx->in == PACT_BF16, st);
-  launch_score_select(bt, true, false, st);
+  launch_prepass(bt, img->N, ctx->in == PACT_BF16, st);
+  launch_logits(bt, img->N, ctx->in == PACT_BF16, st);
+  launch_scores(bt, img->N, st);
   ctx->launches += 3;
   CK(cudaGetLastError());
   return PACT_OK;
@@ -315,7 +329,7 @@ pact_status pact_prune(pact_ctx *ctx, const float *score, int N, const pact_para
   point_counts_at_workspace(m);
   m.score = const_cast<float *>(score);
   m.keep = keep; m.kept_idx = kept_idx; m.pruned_idx = pruned_idx;
-  launch_score_select(bt, false, true, st);
+  launch_select_gather(bt, N, true, false, st);
   ctx->launches += 1;
   CK(cudaGetLastError());
   CK(cudaMemcpyAsync(counts, m.cnt + PACT_CNT_Q, sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
@@ -421,8 +435,11 @@ pact_status pact_merge(pact_ctx *ctx, const pact_image *img, const int32_t *labe
   m.label = const_cast<int32_t *>(label);
   m.C_ptr = C_dev; m.cidx_ptr = center_idx;
   CK(cudaMemsetAsync(m.cnt, 0, 32 * sizeof(int32_t), st));
-  launch_merge(bt, ctx->in == PACT_BF16, ctx->out == PACT_BF16, ctx->ccfg, st);
-  ctx->launches += 1;
+  CK(cudaMemsetAsync(m.csize, 0, (size_t)m.Np * sizeof(int32_t), st));
+  CK(cudaMemsetAsync(m.cticket, 0, (size_t)m.Np * sizeof(int32_t), st));
+  launch_lists(bt, img->N, st);
+  launch_merge(bt, img->N, ctx->in == PACT_BF16, ctx->out == PACT_BF16, ctx->ccfg, st);
+  ctx->launches += 2;
   CK(cudaGetLastError());
   CK(cudaMemcpyAsync(img->counters, m.cnt, sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
   return PACT_OK;
@@ -469,10 +486,10 @@ pact_status pact_reduce(pact_ctx *ctx, const pact_image *imgs, int B, const pact
       return cudaEventRecord(ctx->ev[stage], st);
     };
     if (ctx->prof_on && b0 == 0) CK(cudaEventRecord(ctx->ev[0], st));
-    launch_qsum(bt, cmaxN, bf, st);                 CK(mark());
-    launch_logit_norm(bt, cmaxN, bf, st);           CK(mark());
-    launch_score_select(bt, true, true, st);        CK(mark());
-    launch_keynorm_gather(bt, cmaxN, bf, true, st); CK(mark());
+    launch_prepass(bt, cmaxN, bf, st);              CK(mark());
+    launch_logits(bt, cmaxN, bf, st);               CK(mark());
+    launch_scores(bt, cmaxN, st);                   CK(mark());
+    launch_select_gather(bt, cmaxN, bf, true, st);  CK(mark());
     if (ctx->umma) CK(launch_gram_umma(bt, cmaxN, ctx->ccfg, st));
     else launch_gram(bt, cmaxN, bf, ctx->ccfg, st);
     CK(mark());
@@ -483,12 +500,58 @@ pact_status pact_reduce(pact_ctx *ctx, const pact_image *imgs, int B, const pact
     else launch_assign(bt, cmaxN, bf, ROWS_ALL, ctx->ccfg, st);
     CK(mark());
     launch_label(bt, cmaxN, bf, ROWS_ALL, st);      CK(mark());
-    launch_merge(bt, bf, ctx->out == PACT_BF16, ctx->ccfg, st);  CK(mark());
-    ctx->launches += 11;
+    launch_lists(bt, cmaxN, st);                    CK(mark());
+    launch_merge(bt, cmaxN, bf, ctx->out == PACT_BF16, ctx->ccfg, st);  CK(mark());
+    ctx->launches += 12;
     CK(cudaGetLastError());
     for (int b = 0; b < nb; ++b)
       CK(cudaMemcpyAsync(bt.img[b].counters_user, bt.img[b].cnt, PACT_N_COUNTERS * sizeof(int32_t),
                          cudaMemcpyDeviceToDevice, st));
+  }
+  return PACT_OK;
+}
+
+pact_status pact_graph_create(pact_ctx *ctx, const pact_image *imgs, int B, const pact_params *params,
+                              int params_stride, void *ws, size_t ws_bytes, pact_graph **out) {
+  if (!ctx || !out) return PACT_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (ctx->prof_on) return PACT_ERR_INVALID_ARG;      // per-kernel events are not recorded into graphs
+  cudaStream_t cs = nullptr;
+  CK(cudaStreamCreateWithFlags(&cs, cudaStreamNonBlocking));
+  cudaError_t e = cudaStreamBeginCapture(cs, cudaStreamCaptureModeThreadLocal);
+  if (e != cudaSuccess) { cudaStreamDestroy(cs); return fail_cuda(ctx, e, "cudaStreamBeginCapture"); }
+  const long long before = ctx->launches;
+  const pact_status s = pact_reduce(ctx, imgs, B, params, params_stride, ws, ws_bytes, cs);
+  const int kernels = (int)(ctx->launches - before);
+  ctx->launches = before;                              // nothing has run
+  cudaGraph_t g = nullptr;
+  e = cudaStreamEndCapture(cs, &g);
+  cudaStreamDestroy(cs);
+  if (s != PACT_OK) { if (g) cudaGraphDestroy(g); return s; }
+  if (e != cudaSuccess || !g) return fail_cuda(ctx, e, "cudaStreamEndCapture");
+  cudaGraphExec_t exec = nullptr;
+  e = cudaGraphInstantiate(&exec, g, 0);
+  cudaGraphDestroy(g);
+  if (e != cudaSuccess) return fail_cuda(ctx, e, "cudaGraphInstantiate");
+  pact_graph *pg = new (std::nothrow) pact_graph;
+  if (!pg) { cudaGraphExecDestroy(exec); return PACT_ERR_INVALID_ARG; }
+  pg->ctx = ctx; pg->exec = exec; pg->kernels = kernels;
+  *out = pg;
+  return PACT_OK;
+}
+
+pact_status pact_graph_launch(pact_graph *graph, void *stream) {
+  if (!graph) return PACT_ERR_INVALID_ARG;
+  pact_ctx *ctx = graph->ctx;
+  CK(cudaGraphLaunch(graph->exec, (cudaStream_t)stream));
+  ctx->launches += graph->kernels;
+  return PACT_OK;
+}
+
+pact_status pact_graph_destroy(pact_graph *graph) {
+  if (graph) {
+    cudaGraphExecDestroy(graph->exec);
+    delete graph;
   }
   return PACT_OK;
 }

@@ -14,16 +14,6 @@ __device__ __forceinline__ uint32_t ld_relaxed_u32(const uint32_t *p) {
   return v;
 }
 
-template <typename D> __device__ __forceinline__ typename D::rn_t *rn_tok(const ImgDesc &im);
-template <> __device__ __forceinline__ float *rn_tok<DistF>(const ImgDesc &im) { return im.rn; }
-template <> __device__ __forceinline__ double *rn_tok<DistD>(const ImgDesc &im) { return im.rn64; }
-template <typename D> __device__ __forceinline__ typename D::rn_t *rn_kept(const ImgDesc &im);
-template <> __device__ __forceinline__ float *rn_kept<DistF>(const ImgDesc &im) { return im.rnk; }
-template <> __device__ __forceinline__ double *rn_kept<DistD>(const ImgDesc &im) { return im.rnk64; }
-template <typename D> __device__ __forceinline__ typename D::rn_t *rn_cen(const ImgDesc &im);
-template <> __device__ __forceinline__ float *rn_cen<DistF>(const ImgDesc &im) { return im.rnc; }
-template <> __device__ __forceinline__ double *rn_cen<DistD>(const ImgDesc &im) { return im.rnc64; }
-
 // ---- inverse key norms, survivor gather, per-call initialisation -----------------------------
 // grid (ceil(maxN / 8), B), 256 threads, one warp per work item.
 //  all_tokens = 1: item = token i (inverse norm of every token; survivors are copied to Kp[slot])

@@ -31,11 +31,10 @@ struct ImgDesc {
   double d_c64, inv_dn64, t_reinc64;
   unsigned flags;
   // workspace
-  double *qpart;         // [G][n_qcols] partial column sums of Q
+  double *qpart;         // [kQPartRows][n_qcols] partial column sums of Q
   double *qg;            // [n_qcols] global query
   double *E;             // [N][n_qh] exp(logit - CTA max)
   double *part;          // [G][n_qh][2] per-CTA (max, sum)
-  double *fac;           // [G][n_qh] exp(CTA max - max) / (Z n_qh)
   double *nrm;           // [N] hidden-state norms
   float *score;          // [N]
   unsigned char *keep;   // [N]
@@ -60,7 +59,13 @@ struct ImgDesc {
   int32_t *cid;          // [Np] cluster id of survivor r if it is a centre
   unsigned long long *best;  // [N] packed (distance bits << 32 | cluster id)
   int32_t *label;        // [N]
-  int32_t *cnt;          // [PACT_N_COUNTERS] + scratch: [16] qsum ticket, [17] logit ticket
+  int32_t *blocklist;    // [ceil(N/256)][256] tokens of each block sorted by (cluster id, token)
+  uint16_t *bstart;      // [ceil(N/256)][bstride] tokens of the block with a cluster id below c
+  int32_t *csize;        // [Np] members of cluster c
+  int32_t *cbase;        // [Np] first scratch row of the clusters that are summed in several chunks
+  int32_t *cticket;      // [Np] chunks of cluster c that are finished
+  float *mpart;          // [N/8 + 2][d] chunk sums
+  int32_t *cnt;          // [PACT_N_COUNTERS] + tickets: [16] global query, [19] member lists
   const int32_t *q_ptr;  // where the number of survivors lives (cnt[Q] or the caller's q_dev)
   const int32_t *m_ptr;  // where the number of pruned tokens lives
   const int32_t *C_ptr;  // where the number of clusters lives
@@ -68,6 +73,7 @@ struct ImgDesc {
   float *rho_user;       // optional outputs of the stage calls
   int32_t *center_idx_user, *C_user, *r_user;
   int Np, Wp;            // padded survivor capacity and words per adjacency row
+  int bstride;           // entries per row of bstart
 };
 
 struct Batch {
@@ -108,26 +114,61 @@ __device__ __forceinline__ double warp_sum(double v) {
   return v;
 }
 
-// Sum of squares of one row: each 16-byte vector is summed in float (the squares of bf16
-// values are exact in float), the vectors are accumulated in double.
+// Widens a 16-byte vector that is already in registers.
+template <typename T> __device__ __forceinline__ void widen_vec(const uint4 &v, float (&out)[Vec<T>::N]);
+template <> __device__ __forceinline__ void widen_vec<__nv_bfloat16>(const uint4 &v, float (&out)[8]) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    out[2 * i] = __uint_as_float(w[i] << 16);
+    out[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+  }
+}
+template <> __device__ __forceinline__ void widen_vec<float>(const uint4 &v, float (&out)[4]) {
+  out[0] = __uint_as_float(v.x); out[1] = __uint_as_float(v.y);
+  out[2] = __uint_as_float(v.z); out[3] = __uint_as_float(v.w);
+}
+
+// Sum of squares of 16-byte vectors: each vector is summed in float (the squares of bf16 values are
+// exact in float) and the vectors are accumulated in double.
+template <typename T> __device__ __forceinline__ void sumsq_accumulate(const uint4 &v, double &acc) {
+  constexpr int V = Vec<T>::N;
+  float x[V];
+  widen_vec<T>(v, x);
+  if (sizeof(T) == 2) {
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < V; ++i) s = fmaf(x[i], x[i], s);
+    acc += (double)s;
+  } else {
+#pragma unroll
+    for (int i = 0; i < V; ++i) acc = fma((double)x[i], (double)x[i], acc);
+  }
+}
+
+// This lane's share (vectors lane, lane + 32, ... in ascending order) of the sum of squares of a
+// row of n elements, starting at vector `from`.  Up to U loads per lane are in flight at once.
+template <typename T, int U>
+__device__ __forceinline__ double row_sumsq_lane(const T *row, int n, int lane, int from = 0) {
+  const int nv = n / Vec<T>::N;
+  const uint4 *p = reinterpret_cast<const uint4 *>(row);
+  double acc = 0.0;
+  for (int v0 = from + lane; v0 < nv; v0 += 32 * U) {
+    uint4 buf[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+      if (v0 + 32 * u < nv) buf[u] = __ldg(p + v0 + 32 * u);
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+      if (v0 + 32 * u < nv) sumsq_accumulate<T>(buf[u], acc);
+  }
+  return acc;
+}
+
+// Sum of squares of one row by one warp.
 template <typename T>
 __device__ __forceinline__ double row_sumsq(const T *row, int n, int lane) {
-  constexpr int V = Vec<T>::N;
-  double acc = 0.0;
-  for (int v = lane; v * V < n; v += 32) {
-    float x[V];
-    load_vec<T>(row + (size_t)v * V, x);
-    if (sizeof(T) == 2) {
-      float s = 0.f;
-#pragma unroll
-      for (int i = 0; i < V; ++i) s = fmaf(x[i], x[i], s);
-      acc += (double)s;
-    } else {
-#pragma unroll
-      for (int i = 0; i < V; ++i) acc = fma((double)x[i], (double)x[i], acc);
-    }
-  }
-  return warp_sum(acc);
+  return warp_sum(row_sumsq_lane<T, 8>(row, n, lane));
 }
 
 // ---- distance epilogue: the one place that turns a dot product into a distance ------------
@@ -165,6 +206,16 @@ struct DistD {   // fp32 inputs: double arithmetic
   __device__ static __forceinline__ bool below_t(double d, const ImgDesc &im) { return d < im.t_reinc64; }
   __device__ static __forceinline__ bool in_band_t(double d, const ImgDesc &im) { return fabs(d - im.t_reinc64) <= 1e-6; }
 };
+
+template <typename D> __device__ __forceinline__ typename D::rn_t *rn_tok(const ImgDesc &im);
+template <> __device__ __forceinline__ float *rn_tok<DistF>(const ImgDesc &im) { return im.rn; }
+template <> __device__ __forceinline__ double *rn_tok<DistD>(const ImgDesc &im) { return im.rn64; }
+template <typename D> __device__ __forceinline__ typename D::rn_t *rn_kept(const ImgDesc &im);
+template <> __device__ __forceinline__ float *rn_kept<DistF>(const ImgDesc &im) { return im.rnk; }
+template <> __device__ __forceinline__ double *rn_kept<DistD>(const ImgDesc &im) { return im.rnk64; }
+template <typename D> __device__ __forceinline__ typename D::rn_t *rn_cen(const ImgDesc &im);
+template <> __device__ __forceinline__ float *rn_cen<DistF>(const ImgDesc &im) { return im.rnc; }
+template <> __device__ __forceinline__ double *rn_cen<DistD>(const ImgDesc &im) { return im.rnc64; }
 
 template <typename T> struct DistOf;
 template <> struct DistOf<__nv_bfloat16> { using type = DistF; };

@@ -1,6 +1,17 @@
-// EUTI (Algorithm 1): global query, per-head softmax over the visual tokens, hidden-state norm,
-// percentile split.  All accumulations that decide an ordering are carried in double so that the
-// float32 score the library returns is the correctly rounded value in all but rare cases.
+// EUTI (Algorithm 1): global query (Eq. 1), per-head softmax over the visual tokens and hidden-state
+// norm (Eq. 2), percentile split (Eq. 3-4).  Every accumulation that decides an ordering is carried
+// in double so that the float32 score the library returns is the correctly rounded value in all but
+// rare double-rounding cases.
+//
+//   k_prepass        one pass over Q, H and the clustering keys: column sums of Q -> global query,
+//                    hidden-state norms, inverse key norms (HBM-bound, the only full read of H)
+//   k_logits         k_i . Qglobal per head, CTA-local softmax pieces (max, sum of exp)
+//   k_scores         merges the pieces, writes the float32 scores
+//   k_select_gather  every CTA selects the threshold and compacts (identical results in every CTA),
+//                    then writes its share of the lists and gathers its share of the survivor keys
+//
+// The kernels are short chains of dependent memory round trips; each issues all the loads it can
+// before it consumes the first.
 #include "kernels.cuh"
 
 namespace pact {
@@ -11,33 +22,83 @@ __device__ __forceinline__ double ld_cg_f64(const double *p) {
   return v;
 }
 
-// ---- Eq. 1: column sums of Q ---------------------------------------------------------------
-// grid (G, B), 256 threads; CTA g of image b reduces rows [32g, 32g+32) and the last CTA to
-// finish adds the partial sums in a fixed order.
+constexpr int kPreThreads = 512;
+constexpr int kTokWarps = kPreThreads / 32;   // tokens per CTA of the token part of k_prepass
+constexpr int kQCtasMax = kQPartRows;         // CTAs that reduce Q
+
+// ---- Eq. 1 and the norms -----------------------------------------------------------------------
+// grid (GQ + ceil(maxN / 16), B), 512 threads.
+//  CTAs [0, GQ): column sums of a contiguous block of rows of Q; the last of them to finish adds
+//                the GQ partial sums in index order and writes the global query.
+//  other CTAs:   one warp per visual token: |h_i| (double) and 1 / |k_i| of the clustering key.
 template <typename T>
-__global__ void __launch_bounds__(256) k_qsum(const __grid_constant__ Batch bt) {
-  const ImgDesc &im = bt.img[blockIdx.y];
+__global__ void __launch_bounds__(kPreThreads) k_prepass(const __grid_constant__ Batch bt, int GQ) {
+  using D = typename DistOf<T>::type;
+  using rn_t = typename D::rn_t;
   constexpr int V = Vec<T>::N;
-  const int g = blockIdx.x, t = threadIdx.x;
-  const int G = (im.N + kRowsPerCta - 1) / kRowsPerCta;
-  if (g >= G) return;
-  const int r0 = g * kRowsPerCta, r1 = min(im.N, r0 + kRowsPerCta);
+  const ImgDesc &im = bt.img[blockIdx.y];
+  const int t = threadIdx.x, lane = t & 31, w = t >> 5;
+  if ((int)blockIdx.x >= GQ) {
+    const int tok = ((int)blockIdx.x - GQ) * kTokWarps + w;
+    if (tok >= im.N) return;
+    // every load of the token (key row, then hidden-state row) is issued before the first is used
+    constexpr int UK = 4;
+    const T *krow = im.Kc ? reinterpret_cast<const T *>(im.Kc) + (size_t)tok * im.ldKc : nullptr;
+    const int nvk = krow ? bt.d_k / V : 0;
+    uint4 kb[UK];
+#pragma unroll
+    for (int u = 0; u < UK; ++u)
+      if (lane + 32 * u < nvk) kb[u] = __ldg(reinterpret_cast<const uint4 *>(krow) + lane + 32 * u);
+    if (im.H) {
+      double nn = 1.0;
+      if (!(im.flags & PACT_FLAG_NO_NORM)) {
+        const T *hrow = reinterpret_cast<const T *>(im.H) + (size_t)(im.vis_start + tok) * im.ldH;
+        nn = sqrt(warp_sum(row_sumsq_lane<T, 16>(hrow, bt.d, lane)));
+      }
+      if (lane == 0) im.nrm[tok] = nn;
+    }
+    if (krow) {
+      double acc = 0.0;
+#pragma unroll
+      for (int u = 0; u < UK; ++u)
+        if (lane + 32 * u < nvk) sumsq_accumulate<T>(kb[u], acc);
+      if (nvk > 32 * UK) acc += row_sumsq_lane<T, 8>(krow, bt.d_k, lane, 32 * UK);
+      const double ss = warp_sum(acc);
+      if (lane == 0) rn_tok<D>(im)[tok] = (rn_t)(1.0 / sqrt(fmax(ss, 1e-40)));
+    }
+    return;
+  }
+  if (!im.Q) return;
+  const int g = blockIdx.x;
+  const int chunk = (im.N + GQ - 1) / GQ;
+  const int r0 = min(im.N, g * chunk), r1 = min(im.N, r0 + chunk);
   const int ncolv = bt.n_qcols / V;
-  const int cpp = min(ncolv, 256);          // column vectors per pass
-  const int groups = 256 / cpp;
-  __shared__ double sm[256 * V];
+  const int cpp = min(ncolv, kPreThreads);   // column vectors per pass
+  const int groups = kPreThreads / cpp;      // row groups per pass
+  __shared__ double sm[kPreThreads * V];
   const T *Q = reinterpret_cast<const T *>(im.Q);
+  const int c = t % cpp, gi = t / cpp;
+  constexpr int UQ = 8;
   for (int cbase = 0; cbase < ncolv; cbase += cpp) {
-    const int c = t % cpp, gi = t / cpp;
     double acc[V];
 #pragma unroll
     for (int k = 0; k < V; ++k) acc[k] = 0.0;
     if (gi < groups && cbase + c < ncolv) {
-      for (int r = r0 + gi; r < r1; r += groups) {
-        float x[V];
-        load_vec<T>(Q + (size_t)r * im.ldQ + (size_t)(cbase + c) * V, x);
+      const size_t coff = (size_t)(cbase + c) * V;
+      for (int r = r0 + gi; r < r1; r += groups * UQ) {
+        uint4 buf[UQ];
 #pragma unroll
-        for (int k = 0; k < V; ++k) acc[k] += (double)x[k];
+        for (int u = 0; u < UQ; ++u)
+          if (r + u * groups < r1) buf[u] = __ldg(reinterpret_cast<const uint4 *>(Q + (size_t)(r + u * groups) * im.ldQ + coff));
+#pragma unroll
+        for (int u = 0; u < UQ; ++u) {
+          if (r + u * groups < r1) {
+            float x[V];
+            widen_vec<T>(buf[u], x);
+#pragma unroll
+            for (int k = 0; k < V; ++k) acc[k] += (double)x[k];
+          }
+        }
       }
     }
 #pragma unroll
@@ -55,24 +116,28 @@ __global__ void __launch_bounds__(256) k_qsum(const __grid_constant__ Batch bt) 
   }
   __shared__ int last;
   __threadfence();
-  if (t == 0) last = (atomicAdd(&im.cnt[16], 1) == G - 1);
+  __syncthreads();
+  if (t == 0) last = (atomicAdd(&im.cnt[16], 1) == GQ - 1);
   __syncthreads();
   if (!last) return;
   __threadfence();
-  for (int col = t; col < bt.n_qcols; col += 256) {
+  for (int col = t; col < bt.n_qcols; col += kPreThreads) {
     double s = 0.0;
-    for (int h = 0; h < G; ++h) s += ld_cg_f64(&im.qpart[(size_t)h * bt.n_qcols + col]);
+#pragma unroll 8
+    for (int h = 0; h < GQ; ++h) s += ld_cg_f64(&im.qpart[(size_t)h * bt.n_qcols + col]);
     im.qg[col] = s / (double)im.N;
   }
   if (t == 0) im.cnt[16] = 0;
 }
 
-// ---- Eq. 2, first half: logits, CTA-local softmax pieces, hidden-state norms -----------------
-// grid (G, B), 256 threads, dynamic smem (n_qcols + 32 n_qh) doubles.  One warp per token.
+// ---- Eq. 2, first half: logits and CTA-local softmax pieces ---------------------------------------
+// grid (ceil(maxN / 32), B), 1024 threads, dynamic smem (n_qcols + 32 n_qh) doubles.  One warp per
+// token: the whole key row is loaded at once, then every head takes its part of it.
 template <typename T>
-__global__ void __launch_bounds__(256) k_logit_norm(const __grid_constant__ Batch bt) {
+__global__ void __launch_bounds__(1024) k_logits(const __grid_constant__ Batch bt) {
   const ImgDesc &im = bt.img[blockIdx.y];
   constexpr int V = Vec<T>::N;
+  constexpr int UK = 4;
   const int g = blockIdx.x, t = threadIdx.x, lane = t & 31, w = t >> 5;
   const int G = (im.N + kRowsPerCta - 1) / kRowsPerCta;
   if (g >= G) return;
@@ -80,204 +145,355 @@ __global__ void __launch_bounds__(256) k_logit_norm(const __grid_constant__ Batc
   double *qg = smd;                       // [n_qcols]
   double *lg = smd + bt.n_qcols;          // [32][n_qh]
   const int n_qh = bt.n_qh, d_h = bt.d_h;
-  for (int c = t; c < bt.n_qcols; c += 256) qg[c] = ld_cg_f64(&im.qg[c]);
-  __syncthreads();
   const int r0 = g * kRowsPerCta, r1 = min(im.N, r0 + kRowsPerCta);
-  const T *H = reinterpret_cast<const T *>(im.H);
-  const T *K = reinterpret_cast<const T *>(im.Ke);
-  const bool use_norm = !(im.flags & PACT_FLAG_NO_NORM);
   const bool use_query = !(im.flags & PACT_FLAG_NORM_ONLY);
-  for (int r = r0 + w; r < r1; r += 8) {
-    double nn = 1.0;
-    if (use_norm) nn = sqrt(row_sumsq<T>(H + (size_t)(im.vis_start + r) * im.ldH, bt.d, lane));
-    if (lane == 0) im.nrm[r] = nn;
+  const int r = r0 + w;
+  const int nv = bt.d_k / V;
+  const uint4 *krow = reinterpret_cast<const uint4 *>(reinterpret_cast<const T *>(im.Ke) + (size_t)min(r, im.N - 1) * im.ldKe);
+  uint4 kb[UK];
+  if (use_query) {
+#pragma unroll
+    for (int u = 0; u < UK; ++u)
+      if (lane + 32 * u < nv) kb[u] = __ldg(krow + lane + 32 * u);
+  }
+  for (int c = t; c < bt.n_qcols; c += 1024) qg[c] = im.qg[c];
+  __syncthreads();
+  if (r < r1) {
     for (int j = 0; j < n_qh; ++j) {
       double acc = 0.0;
       if (use_query) {
         const int kv = (j * bt.n_kvh) / n_qh;
-        const T *kr = K + (size_t)r * im.ldKe + (size_t)kv * d_h;
-        const double *qr = qg + (size_t)j * d_h;
-        for (int v = lane; v * V < d_h; v += 32) {
-          float x[V];
-          load_vec<T>(kr + v * V, x);
+        const double *qr = qg + (size_t)j * d_h - (size_t)kv * d_h;    // indexed by the element's place in the row
 #pragma unroll
-          for (int k = 0; k < V; ++k) acc = fma((double)x[k], qr[v * V + k], acc);
+        for (int u = 0; u < UK; ++u) {
+          const int e0 = (lane + 32 * u) * V;
+          if (lane + 32 * u < nv && e0 / d_h == kv) {
+            float x[V];
+            widen_vec<T>(kb[u], x);
+#pragma unroll
+            for (int k = 0; k < V; ++k) acc = fma((double)x[k], qr[e0 + k], acc);
+          }
+        }
+        for (int v = lane + 32 * UK; v < nv; v += 32) {               // rows wider than the preloaded part
+          const int e0 = v * V;
+          if (e0 / d_h == kv) {
+            float x[V];
+            widen_vec<T>(__ldg(krow + v), x);
+#pragma unroll
+            for (int k = 0; k < V; ++k) acc = fma((double)x[k], qr[e0 + k], acc);
+          }
         }
         acc = warp_sum(acc);
       }
-      if (lane == 0) lg[(r - r0) * n_qh + j] = acc;
+      if (lane == 0) lg[w * n_qh + j] = acc;
     }
   }
   __syncthreads();
   // per head: CTA max, exp, CTA sum; lane = token within the CTA
-  for (int j = w; j < n_qh; j += 8) {
-    const int r = r0 + lane;
-    const bool ok = r < r1;
-    double l = ok ? lg[lane * n_qh + j] : -1.0e300;
+  for (int j = w; j < n_qh; j += 32) {
+    const int rr = r0 + lane;
+    const bool ok = rr < r1;
+    const double l = ok ? lg[lane * n_qh + j] : -1.0e300;
     double m = l;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m = fmax(m, __shfl_xor_sync(0xffffffffu, m, o));
-    double e = ok ? exp(l - m) : 0.0;
-    if (ok) im.E[(size_t)r * n_qh + j] = e;
-    double s = warp_sum(e);
+    const double e = ok ? exp(l - m) : 0.0;
+    if (ok) im.E[(size_t)rr * n_qh + j] = e;
+    const double s = warp_sum(e);
     if (lane == 0) {
       im.part[((size_t)g * n_qh + j) * 2] = m;
       im.part[((size_t)g * n_qh + j) * 2 + 1] = s;
     }
   }
-  __shared__ int last;
-  __shared__ double red[8];
-  __threadfence();
-  __syncthreads();
-  if (t == 0) last = (atomicAdd(&im.cnt[17], 1) == G - 1);
-  __syncthreads();
-  if (!last) return;
-  __threadfence();
-  // merge the CTA pieces in a fixed order: M = max, Z = sum S_g exp(M_g - M)
-  for (int j = 0; j < n_qh; ++j) {
-    double m = -1.0e300;
-    for (int h = t; h < G; h += 256) m = fmax(m, ld_cg_f64(&im.part[((size_t)h * n_qh + j) * 2]));
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) m = fmax(m, __shfl_xor_sync(0xffffffffu, m, o));
-    if (lane == 0) red[w] = m;
-    __syncthreads();
-    m = red[0];
-    for (int k = 1; k < 8; ++k) m = fmax(m, red[k]);
-    __syncthreads();
-    double z = 0.0;
-    for (int h = t; h < G; h += 256) {
-      double wgt = exp(ld_cg_f64(&im.part[((size_t)h * n_qh + j) * 2]) - m);
-      im.fac[(size_t)h * n_qh + j] = wgt;
-      z += ld_cg_f64(&im.part[((size_t)h * n_qh + j) * 2 + 1]) * wgt;
-    }
-    z = warp_sum(z);
-    if (lane == 0) red[w] = z;
-    __syncthreads();
-    z = 0.0;
-    for (int k = 0; k < 8; ++k) z += red[k];
-    __syncthreads();
-    const double inv = 1.0 / (z * (double)n_qh);
-    for (int h = t; h < G; h += 256) im.fac[(size_t)h * n_qh + j] *= inv;
-  }
-  if (t == 0) im.cnt[17] = 0;
 }
 
-// ---- Eq. 2 second half and Eq. 3-4: scores, order statistic, ordered compaction ---------------
-// grid (1, B), 1024 threads.
+// ---- Eq. 2, second half: merge the pieces (M = max, Z = sum S_g exp(M_g - M), fixed order), scores --
+// grid (ceil(maxN / 256), B), 256 threads.  Every CTA merges all pieces itself, one warp per head.
+__global__ void __launch_bounds__(256) k_scores(const __grid_constant__ Batch bt) {
+  const ImgDesc &im = bt.img[blockIdx.y];
+  const int t = threadIdx.x, lane = t & 31, w = t >> 5;
+  const int N = im.N, n_qh = bt.n_qh;
+  if ((int)blockIdx.x * 256 >= N) return;
+  const int G = (N + kRowsPerCta - 1) / kRowsPerCta;
+  __shared__ double sM[256], sInv[256];
+  const int i = blockIdx.x * 256 + t;
+  // this token's terms, requested before the merge so that they arrive meanwhile
+  constexpr int EP = 4;
+  double e_pre[EP], nrm_i = 0.0;
+  const bool pre = n_qh <= EP && i < N;
+  if (pre) {
+#pragma unroll
+    for (int j = 0; j < EP; ++j) e_pre[j] = j < n_qh ? im.E[(size_t)i * n_qh + j] : 0.0;
+  }
+  if (i < N) nrm_i = im.nrm[i];
+  for (int j = w; j < n_qh; j += 8) {
+    const double *pj = im.part + (size_t)j * 2;
+    const size_t stride = (size_t)n_qh * 2;
+    double m = -1.0e300;
+#pragma unroll 4
+    for (int h = lane; h < G; h += 32) m = fmax(m, pj[(size_t)h * stride]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmax(m, __shfl_xor_sync(0xffffffffu, m, o));
+    double z = 0.0;
+#pragma unroll 4
+    for (int h = lane; h < G; h += 32) z += pj[(size_t)h * stride + 1] * exp(pj[(size_t)h * stride] - m);
+    z = warp_sum(z);
+    if (lane == 0) { sM[j] = m; sInv[j] = 1.0 / (z * (double)n_qh); }
+  }
+  __syncthreads();
+  if (i >= N) return;
+  const int g = i / kRowsPerCta;
+  double s = 0.0;
+  for (int j = 0; j < n_qh; ++j) {
+    const double fac = exp(im.part[((size_t)g * n_qh + j) * 2] - sM[j]) * sInv[j];
+    double e;
+    if (pre) {
+      e = e_pre[0];
+#pragma unroll
+      for (int q = 1; q < EP; ++q) if (j == q) e = e_pre[q];
+    } else {
+      e = im.E[(size_t)i * n_qh + j];
+    }
+    s = fma(e, fac, s);
+  }
+  const float sf = (float)(s * nrm_i);
+  im.score[i] = sf;
+  if (im.score_user) im.score_user[i] = sf;
+}
+
+// ---- Eq. 3-4: order statistic, ordered compaction; survivor key gather ------------------------------
 __device__ __forceinline__ uint32_t score_key(float s) {
   uint32_t b = __float_as_uint(s);
   if (b == 0x80000000u) b = 0;                       // -0 orders as +0
   return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
-__global__ void __launch_bounds__(1024) k_score_select(const __grid_constant__ Batch bt, int do_score,
-                                                       int do_select) {
+// grid (X, B), 1024 threads; dynamic smem: (keys_in_smem) N keys, then own_cap token indices.
+// Every CTA computes the same threshold and the same list positions; CTA b writes the list entries of
+// its block of tokens, and (do_gather) copies its block of survivor rows into Kp and their inverse
+// norms into rnk, and clears its share of the arrays that later kernels accumulate into.
+template <typename T>
+__global__ void __launch_bounds__(1024) k_select_gather(const __grid_constant__ Batch bt, int do_gather,
+                                                        int keys_in_smem, int own_cap) {
+  using D = typename DistOf<T>::type;
   const ImgDesc &im = bt.img[blockIdx.y];
   const int t = threadIdx.x, lane = t & 31, w = t >> 5;
-  const int N = im.N, n_qh = bt.n_qh;
+  const int N = im.N;
+  extern __shared__ uint32_t dsm[];
+  uint32_t *skey = dsm;                                     // [N] when keys_in_smem
+  int *own = reinterpret_cast<int *>(dsm + (keys_in_smem ? N : 0));   // [own_cap]
   __shared__ int hist[256];
   __shared__ int warp_tot[32];
   __shared__ uint32_t s_prefix;
-  __shared__ int s_k, s_running;
-  if (do_score) {
-    for (int i = t; i < N; i += 1024) {
-      const int g = i / kRowsPerCta;
-      double s = 0.0;
-      for (int j = 0; j < n_qh; ++j) s = fma(im.E[(size_t)i * n_qh + j], im.fac[(size_t)g * n_qh + j], s);
-      const float sf = (float)(s * im.nrm[i]);
-      im.score[i] = sf;
-      if (im.score_user) im.score_user[i] = sf;
-    }
-    __syncthreads();
+  __shared__ int s_k;
+
+  if (keys_in_smem)
+    for (int i = t; i < N; i += 1024) skey[i] = score_key(im.score[i]);
+  if (do_gather) {   // per-call initialisation, spread over the grid
+    const int gt = blockIdx.x * 1024 + t, gs = gridDim.x * 1024;
+    for (int r = gt; r < im.Np; r += gs) { im.rho_fix[r] = 0ull; im.rank[r] = 0; im.csize[r] = 0; im.cticket[r] = 0; }
+    for (int wd = gt; wd < im.Wp; wd += gs) { im.cmask[wd] = 0u; im.rmask[wd] = 0u; }
+    for (int i = gt; i < N; i += gs) im.best[i] = kBestInit;
   }
-  if (!do_select) return;
-  // radix select of the (m_target + 1)-th smallest key, most significant byte first
   if (t == 0) { s_prefix = 0; s_k = im.m_target; }
+  if (t < 256) hist[t] = 0;
+  __syncthreads();
+  auto key = [&](int i) -> uint32_t { return keys_in_smem ? skey[i] : score_key(im.score[i]); };
+
+  // radix select of the (m_target + 1)-th smallest key, most significant byte first; lanes of a
+  // warp that hit the same bin add once
   uint32_t mask = 0;
+  const int rounds = (N + 1023) / 1024;
   for (int pass = 3; pass >= 0; --pass) {
     const int shift = pass * 8;
-    if (t < 256) hist[t] = 0;
-    __syncthreads();
     const uint32_t prefix = s_prefix;
-    for (int i = t; i < N; i += 1024) {
-      const uint32_t key = score_key(im.score[i]);
-      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255], 1);
+    for (int it = 0; it < rounds; ++it) {
+      const int i = it * 1024 + t;
+      bool valid = i < N;
+      uint32_t kk = 0;
+      if (valid) { kk = key(i); valid = (kk & mask) == prefix; }
+      const uint32_t dgt = (kk >> shift) & 255u;
+      const unsigned peers = __match_any_sync(0xffffffffu, valid ? dgt : (256u + lane));
+      if (valid && lane == __ffs(peers) - 1) atomicAdd(&hist[dgt], __popc(peers));
     }
     __syncthreads();
-    if (t == 0) {
-      int k = s_k, dgt = 0;
-      while (dgt < 255 && k >= hist[dgt]) { k -= hist[dgt]; ++dgt; }
-      s_k = k;
-      s_prefix = prefix | ((uint32_t)dgt << shift);
+    if (w == 0) {
+      int c[8], s = 0;
+#pragma unroll
+      for (int b = 0; b < 8; ++b) { c[b] = hist[lane * 8 + b]; s += c[b]; }
+      int incl = s;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += y;
+      }
+      const int k = s_k;
+      const unsigned has = __ballot_sync(0xffffffffu, incl > k);
+      const int L = has ? __ffs(has) - 1 : 31;   // the candidates always number more than k
+      if (lane == L) {
+        int kk = k - (incl - s), dgt = 7;
+        bool done = false;
+#pragma unroll
+        for (int b = 0; b < 7; ++b) {
+          if (!done) {
+            if (kk < c[b]) { dgt = b; done = true; }
+            else kk -= c[b];
+          }
+        }
+        s_k = kk;
+        s_prefix = prefix | ((uint32_t)(lane * 8 + dgt) << shift);
+      }
+#pragma unroll
+      for (int b = 0; b < 8; ++b) hist[lane * 8 + b] = 0;
     }
     mask |= 255u << shift;
     __syncthreads();
   }
   const uint32_t tau_key = s_prefix;
-  if (t == 0) s_running = 0;
-  __syncthreads();
-  for (int base = 0; base < N; base += 1024) {
-    const int i = base + t;
-    const bool kp = i < N && score_key(im.score[i]) >= tau_key;
-    const unsigned bal = __ballot_sync(0xffffffffu, kp);
-    if (lane == 0) warp_tot[w] = __popc(bal);
-    __syncthreads();
-    if (w == 0) {
-      int v = warp_tot[lane], x = v;
+
+  // ordered compaction: thread t owns tokens [t * CH, t * CH + CH)
+  const int CH = (N + 1023) / 1024;
+  const int i0 = min(N, t * CH), i1 = min(N, i0 + CH);
+  int mine = 0;
+  for (int i = i0; i < i1; ++i) mine += key(i) >= tau_key;
+  int incl = mine;
 #pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        int y = __shfl_up_sync(0xffffffffu, x, o);
-        if (lane >= o) x += y;
-      }
-      warp_tot[lane] = x - v;                          // exclusive
-      if (lane == 31) s_k = x;                         // kept in this chunk
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += y;
+  }
+  if (lane == 31) warp_tot[w] = incl;
+  __syncthreads();
+  if (w == 0) {
+    const int v = warp_tot[lane];
+    int x = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, x, o);
+      if (lane >= o) x += y;
     }
-    __syncthreads();
-    const int before = s_running + warp_tot[w] + __popc(bal & ((1u << lane) - 1u));
-    if (i < N) {
+    warp_tot[lane] = x - v;                                 // exclusive
+    if (lane == 31) s_k = x;                                // q
+  }
+  __syncthreads();
+  const int q = s_k;
+  int before = warp_tot[w] + incl - mine;                   // survivors with a lower index
+  const int tpc = (N + gridDim.x - 1) / gridDim.x;          // tokens whose list entries this CTA writes
+  const int w0 = blockIdx.x * tpc, w1 = min(N, w0 + tpc);
+  const int rpc = (q + gridDim.x - 1) / gridDim.x;          // survivor rows this CTA gathers
+  const int g0 = min(q, (int)blockIdx.x * rpc), g1 = min(q, g0 + rpc);
+  for (int i = i0; i < i1; ++i) {
+    const bool kp = key(i) >= tau_key;
+    if (i >= w0 && i < w1) {
       im.keep[i] = kp ? 1 : 0;
       if (im.keep_user) im.keep_user[i] = kp ? 1 : 0;
       if (kp) { im.kept_idx[before] = i; im.slot[i] = before; }
       else { im.pruned_idx[i - before] = i; im.slot[i] = -1 - (i - before); }
     }
-    __syncthreads();
-    if (t == 0) s_running += s_k;
-    __syncthreads();
+    if (kp) {
+      if (do_gather && before >= g0 && before < g1 && before - g0 < own_cap) own[before - g0] = i;
+      ++before;
+    }
   }
-  if (t == 0) {
-    im.cnt[PACT_CNT_Q] = s_running;
-    im.cnt[PACT_CNT_M] = N - s_running;
+  if (blockIdx.x == 0 && t == 0) {
+    im.cnt[PACT_CNT_Q] = q;
+    im.cnt[PACT_CNT_M] = N - q;
+  }
+  if (!do_gather) return;
+  __syncthreads();
+  constexpr int V = Vec<T>::N;
+  const int nv = bt.d_k / V;
+  const T *Kc = reinterpret_cast<const T *>(im.Kc);
+  T *Kp = reinterpret_cast<T *>(im.Kp);
+  for (int rr = g0 + w; rr < g1; rr += 32) {
+    const int tok = own[rr - g0];
+    const uint4 *src = reinterpret_cast<const uint4 *>(Kc + (size_t)tok * im.ldKc);
+    uint4 *dst = reinterpret_cast<uint4 *>(Kp + (size_t)rr * bt.d_k);
+    for (int v0 = lane; v0 < nv; v0 += 128) {
+      uint4 buf[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (v0 + 32 * u < nv) buf[u] = __ldg(src + v0 + 32 * u);
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (v0 + 32 * u < nv) dst[v0 + 32 * u] = buf[u];
+    }
+    if (lane == 0) rn_kept<D>(im)[rr] = rn_tok<D>(im)[tok];
   }
 }
 
 // ---- launchers -----------------------------------------------------------------------------
 
-void launch_qsum(const Batch &bt, int maxN, bool bf16, cudaStream_t st) {
-  dim3 grid((maxN + kRowsPerCta - 1) / kRowsPerCta, bt.B);
-  if (bf16) k_qsum<__nv_bfloat16><<<grid, 256, 0, st>>>(bt);
-  else k_qsum<float><<<grid, 256, 0, st>>>(bt);
+namespace {
+int g_sm_count = 148;
+size_t g_smem_optin = 48 * 1024;
+constexpr size_t kSelectReserve = 4096;      // static shared memory of k_select_gather, rounded up
+
+int q_ctas(int maxN) {
+  const int g = (maxN + 127) / 128;
+  return g < 1 ? 1 : (g > kQCtasMax ? kQCtasMax : g);
+}
+}  // namespace
+
+void launch_prepass(const Batch &bt, int maxN, bool bf16, cudaStream_t st) {
+  const int GQ = q_ctas(maxN);
+  dim3 grid(GQ + (maxN + kTokWarps - 1) / kTokWarps, bt.B);
+  if (bf16) k_prepass<__nv_bfloat16><<<grid, kPreThreads, 0, st>>>(bt, GQ);
+  else k_prepass<float><<<grid, kPreThreads, 0, st>>>(bt, GQ);
 }
 
-void launch_logit_norm(const Batch &bt, int maxN, bool bf16, cudaStream_t st) {
+void launch_logits(const Batch &bt, int maxN, bool bf16, cudaStream_t st) {
   dim3 grid((maxN + kRowsPerCta - 1) / kRowsPerCta, bt.B);
   const size_t sm = (size_t)(bt.n_qcols + kRowsPerCta * bt.n_qh) * sizeof(double);
-  if (bf16) k_logit_norm<__nv_bfloat16><<<grid, 256, sm, st>>>(bt);
-  else k_logit_norm<float><<<grid, 256, sm, st>>>(bt);
+  if (bf16) k_logits<__nv_bfloat16><<<grid, 1024, sm, st>>>(bt);
+  else k_logits<float><<<grid, 1024, sm, st>>>(bt);
 }
 
-void launch_score_select(const Batch &bt, bool score, bool select, cudaStream_t st) {
-  k_score_select<<<dim3(1, bt.B), 1024, 0, st>>>(bt, score ? 1 : 0, select ? 1 : 0);
+void launch_scores(const Batch &bt, int maxN, cudaStream_t st) {
+  k_scores<<<dim3((maxN + 255) / 256, bt.B), 256, 0, st>>>(bt);
 }
 
-size_t euti_smem_bytes(int n_qcols, int n_qh) {
-  return (size_t)(n_qcols + kRowsPerCta * n_qh) * sizeof(double);
+void launch_select_gather(const Batch &bt, int maxN, bool bf16, bool gather, cudaStream_t st) {
+  int X = 1;
+  if (gather) {
+    X = g_sm_count / bt.B;
+    if (X < 1) X = 1;
+    const int cap = (maxN + 31) / 32;          // at least 32 survivor rows per CTA
+    if (X > cap) X = cap;
+  }
+  const int own_cap = gather ? (maxN + X - 1) / X + 1 : 0;
+  size_t sm = (size_t)own_cap * sizeof(int);
+  const bool in_smem = sm + (size_t)maxN * 4 + kSelectReserve <= g_smem_optin;
+  if (in_smem) sm += (size_t)maxN * 4;
+  dim3 grid(X, bt.B);
+  if (bf16) k_select_gather<__nv_bfloat16><<<grid, 1024, sm, st>>>(bt, gather ? 1 : 0, in_smem ? 1 : 0, own_cap);
+  else k_select_gather<float><<<grid, 1024, sm, st>>>(bt, gather ? 1 : 0, in_smem ? 1 : 0, own_cap);
+}
+
+cudaError_t select_configure() {
+  int dev = 0, v = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  e = cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return e;
+  g_sm_count = v;
+  e = cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  if (e != cudaSuccess) return e;
+  g_smem_optin = (size_t)v;
+  const int dyn = (int)(g_smem_optin - kSelectReserve);
+  e = cudaFuncSetAttribute(k_select_gather<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(k_select_gather<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn);
 }
 
 cudaError_t euti_configure(int n_qcols, int n_qh) {
-  const size_t sm = euti_smem_bytes(n_qcols, n_qh);
-  cudaError_t e = cudaFuncSetAttribute(k_logit_norm<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+  cudaError_t e = select_configure();
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(k_logit_norm<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+  const size_t sm = (size_t)(n_qcols + kRowsPerCta * n_qh) * sizeof(double);
+  if (sm > g_smem_optin) return cudaErrorInvalidConfiguration;
+  e = cudaFuncSetAttribute(k_logits<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(k_logits<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
 }
 
 }  // namespace pact

@@ -10,10 +10,14 @@ constexpr int kMergeMaxD = 256 * 4 * 8;   // widest hidden state the merge kerne
 enum RowMode { ROWS_ALL = 0, ROWS_KEPT_LIST = 1, ROWS_PRUNED_LIST = 2 };
 
 // euti.cu
-void launch_qsum(const Batch &bt, int maxN, bool bf16, cudaStream_t st);
-void launch_logit_norm(const Batch &bt, int maxN, bool bf16, cudaStream_t st);
-void launch_score_select(const Batch &bt, bool score, bool select, cudaStream_t st);
+constexpr int kQPartRows = 32;            // most partial sums of Q the prepass writes per image
+void launch_prepass(const Batch &bt, int maxN, bool bf16, cudaStream_t st);
+void launch_logits(const Batch &bt, int maxN, bool bf16, cudaStream_t st);
+void launch_scores(const Batch &bt, int maxN, cudaStream_t st);
+// threshold + ordered compaction; gather: also copy the survivor keys and clear the accumulators
+void launch_select_gather(const Batch &bt, int maxN, bool bf16, bool gather, cudaStream_t st);
 cudaError_t euti_configure(int n_qcols, int n_qh);
+cudaError_t select_configure();            // what launch_select_gather needs, once per device
 
 // cluster.cu
 struct ClusterCfg {
@@ -38,6 +42,8 @@ cudaError_t launch_gram_umma(const Batch &bt, int maxN, const ClusterCfg &cfg, c
 cudaError_t launch_assign_umma(const Batch &bt, int maxN, bool kept_rows, const ClusterCfg &cfg, cudaStream_t st);
 
 // merge.cu
-void launch_merge(const Batch &bt, bool in_bf16, bool out_bf16, const ClusterCfg &cfg, cudaStream_t st);
+// member lists from label[]; csize and cticket must be zero
+void launch_lists(const Batch &bt, int maxN, cudaStream_t st);
+void launch_merge(const Batch &bt, int maxN, bool in_bf16, bool out_bf16, const ClusterCfg &cfg, cudaStream_t st);
 
 }  // namespace pact

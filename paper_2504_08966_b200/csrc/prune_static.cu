@@ -42,6 +42,8 @@ cudaError_t scratch_for_current_device(void **out) {
     e = cudaGetSymbolAddress(&p, g_prune_scratch);
     if (e != cudaSuccess) return e;
     if (!p) return cudaErrorInvalidSymbol;
+    e = select_configure();
+    if (e != cudaSuccess) return e;
     g_scratch_addr[dev] = p;
   }
   *out = g_scratch_addr[dev];
@@ -76,7 +78,7 @@ extern "C" pact_status pact_prune_static(const float *score, int N, const pact_p
   m.pruned_idx = pruned_idx;
   // The array keeps whatever the previous call left: start the counters from zero.
   if (cudaMemsetAsync(m.cnt, 0, kStaticCntInts * sizeof(int32_t), st) != cudaSuccess) return PACT_ERR_CUDA;
-  launch_score_select(bt, false, true, st);
+  launch_select_gather(bt, N, true, false, st);
   if (cudaGetLastError() != cudaSuccess) return PACT_ERR_CUDA;
   if (cudaMemcpyAsync(counts, m.cnt + PACT_CNT_Q, sizeof(int32_t), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
     return PACT_ERR_CUDA;

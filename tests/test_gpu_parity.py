@@ -157,6 +157,28 @@ def test_bitwise_deterministic_run_to_run():
     assert np.array_equal(a[0]["score"].view(np.int32), b[0]["score"].view(np.int32))
 
 
+def test_graph_replay_matches_direct_call_bitwise():
+    from paper_2504_08966_b200 import binding as pb
+    wl = workloads.single_image(seed=72, N=2100, T=10, n_blobs=50)
+    direct, _ = gpu_reduce(wl, torch.bfloat16)
+    ctx = pb.Context(wl.d, wl.n_qh, wl.n_kvh, wl.d_h, wl.dtype, torch.bfloat16)
+    ims = [pb.device_image(img, torch.bfloat16) for img in wl.images]
+    g = ctx.pact_graph_create(ims, pb.make_params(lam=wl.lam, d_c=wl.d_c, d_n=wl.d_n, alpha=wl.alpha))
+    for rep in range(3):
+        ims[0].H_out.zero_()
+        ims[0].label.fill_(-7)
+        g.launch()
+        torch.cuda.synchronize()
+        cnt = ims[0].counters.cpu().numpy()
+        n_out = int(cnt[pb.CNT["n_out"]])
+        assert int(cnt[pb.CNT["status"]]) == 0 and n_out == direct[0]["n_out"]
+        assert np.array_equal(ims[0].label.cpu().numpy(), direct[0]["label"])
+        assert torch.equal(ims[0].H_out[:n_out].cpu().view(torch.int16), direct[0]["H_out_raw"].view(torch.int16))
+    o = oracle_image(wl, wl.images[0])
+    assert np.array_equal(direct[0]["label"], o["label"])
+    g.close()
+
+
 # ------------------------------------------------------------------ stage calls against the oracle's stages
 
 @pytest.fixture(scope="module")
