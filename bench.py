@@ -171,7 +171,9 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     W = max(3, args.warmup)
 
-    wl = workloads.build(args.workload, seed={"single_image": 1, "video": 3, "batched": 2, "stress": 4}[args.workload] + 100 * rank)
+    from paper_2504_08966_b200 import sharding
+    base_seed = {"single_image": 1, "video": 3, "batched": 2, "stress": 4}[args.workload]
+    wl = workloads.build(args.workload, seed=sharding.rank_seed(base_seed, rank))
     ctx = pb.Context(wl.d, wl.n_qh, wl.n_kvh, wl.d_h, wl.dtype, torch.bfloat16)
     params = pb.make_params(lam=wl.lam, d_c=wl.d_c, d_n=wl.d_n, alpha=wl.alpha)
     n_vis = sum(im.N for im in wl.images)

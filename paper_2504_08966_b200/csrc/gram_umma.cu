@@ -3,10 +3,11 @@
 // nearest-centre pass (Algorithm 2 assignment, Eq. 8).  Nothing of the distance matrix reaches
 // memory: accumulators live in tensor memory and are consumed from there.
 //
-// One persistent CTA per SM, 192 threads:
+// One persistent CTA per SM, 320 threads:
 //   warp 0      TMA producer: 128-byte-swizzled K-slabs of the two operands into a shared-memory ring
 //   warp 1      allocates tensor memory, issues tcgen05.mma (128 x BN x 16, bf16 -> fp32)
-//   warps 2-5   epilogue: tcgen05.ld of their 32-lane quadrant, distance arithmetic of common.cuh
+//   warps 2-9   epilogue: tcgen05.ld of their 32-lane quadrant (two warps per quadrant, half of the
+//               columns each), distance arithmetic of common.cuh
 // Two accumulators (2 x BN columns of tensor memory) let the epilogue of tile t overlap the MMAs of
 // tile t+1.  Every mbarrier wait is bounded; when one runs out the CTA raises the image's status
 // word, drains what it armed, frees its tensor memory and returns.
@@ -121,22 +122,62 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
 // kind::f16 instruction descriptor: fp32 accumulate, bf16 x bf16, both operands K-major.
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
+constexpr int EPI_WARPS = 8;      // two per tensor-memory lane quadrant; each takes half of the columns
+constexpr int THREADS = 64 + EPI_WARPS * 32;
+constexpr int HALF = BN / 2;      // columns per epilogue warp
+
 struct Shared {
   uint64_t full[STAGES], empty[STAGES], acc_full[2], acc_empty[2];
   uint32_t tmem_base;
   int abort;
-  float rn_col[4][BN];          // one copy per epilogue warp
+  __align__(16) float rn_col[EPI_WARPS][HALF];   // inverse norms of this warp's columns
 };
 
 enum { MODE_GRAM = 0, MODE_ASSIGN = 1 };
 
+// One 32-column chunk of the epilogue of the all-pairs pass for one row (= one lane): distance
+// (Eq. 5), density term (Eq. 6) as an integer multiple of 2^-30, adjacency bit d <= d_c, band count.
+// SLOW adds the per-element checks that only edge chunks need (diagonal, columns past the end).
+template <bool SLOW>
+__device__ __forceinline__ void gram_chunk(const uint32_t (&v)[32], const float *rn_col, float rni, int row, int c0,
+                                           int ncols, const ImgDesc &im, unsigned long long &rowsum, uint32_t &bits,
+                                           int &band) {
+  uint32_t b = 0u;
+  unsigned long long s = 0ull;
+#pragma unroll
+  for (int k4 = 0; k4 < 32; k4 += 4) {
+    const float4 rn4 = *reinterpret_cast<const float4 *>(rn_col + k4);
+    const float rnj[4] = {rn4.x, rn4.y, rn4.z, rn4.w};
+#pragma unroll
+    for (int kk = 0; kk < 4; ++kk) {
+      const int k = k4 + kk;
+      float dd = DistF::dist(__uint_as_float(v[k]), rni, rnj[kk]);
+      if (SLOW) {
+        const int gj = c0 + k;
+        if (gj == row) dd = 0.f;
+        if (gj < ncols) {
+          s += DistF::term(dd, im);
+          if (DistF::within(dd, im)) b |= 1u << k;
+          if (row < gj && DistF::in_band(dd, im)) ++band;
+        }
+      } else {
+        s += DistF::term(dd, im);
+        if (DistF::within(dd, im)) b |= 1u << k;
+        if (DistF::in_band(dd, im)) ++band;
+      }
+    }
+  }
+  rowsum += s;
+  bits = b;
+}
+
 }  // namespace
 
-// grid (X, B), 192 threads, dynamic smem = 1024 (alignment slack) + STAGES * STAGE_BYTES.
+// grid (X, B), 320 threads, dynamic smem = 1024 (alignment slack) + STAGES * STAGE_BYTES.
 // kept_rows (assignment only): rows are the gathered survivors (Kp, rnk) instead of all tokens.
 template <int MODE>
-__global__ void __launch_bounds__(192, 1) k_tiles_umma(const __grid_constant__ Batch bt,
-                                                       const __grid_constant__ TmapSet tm, int kept_rows) {
+__global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant__ Batch bt,
+                                                           const __grid_constant__ TmapSet tm, int kept_rows) {
   const ImgDesc &im = bt.img[blockIdx.y];
   extern __shared__ uint8_t smem_raw[];
   __shared__ Shared sh;
@@ -153,7 +194,7 @@ __global__ void __launch_bounds__(192, 1) k_tiles_umma(const __grid_constant__ B
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(&sh.acc_full[a], 1); mbar_init(&sh.acc_empty[a], 4); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&sh.acc_full[a], 1); mbar_init(&sh.acc_empty[a], EPI_WARPS); }
     sh.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -215,72 +256,86 @@ __global__ void __launch_bounds__(192, 1) k_tiles_umma(const __grid_constant__ B
     }
   } else {
     // ---------------- epilogue ----------------
-    const int qd = warp & 3;                        // tensor-memory lane quadrant of this warp
-    float *rn_col = sh.rn_col[qd];
+    const int ew = warp - 2;
+    const int qd = warp & 3;                        // tensor-memory lane quadrant this warp may read
+    const int half = ew >> 2;                       // which half of the tile's columns
+    float *rn_col = sh.rn_col[ew];
     uint32_t tcount = 0;
     int band = 0;
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < ntiles; tile += gridDim.x, ++tcount) {
       const int tmi = tile / ntn, tni = tile % ntn;
       const uint32_t a = tcount & 1;
-      // inverse norms of this tile's columns
-      __syncwarp();
-      for (int c = lane; c < BN; c += 32) {
-        const int gj = tni * BN + c;
-        rn_col[c] = gj < ncols ? (MODE == MODE_GRAM ? im.rnk[gj] : im.rnc[gj]) : 0.f;
+      const int cbase = tni * BN + half * HALF;     // first column of this warp
+      // inverse norms of this warp's columns and of this lane's row (in flight while the MMAs run)
+      const float *rn_src = MODE == MODE_GRAM ? im.rnk : im.rnc;
+      float4 r4;
+      {
+        const int gj = cbase + lane * 4;
+        r4.x = gj + 0 < ncols ? rn_src[gj + 0] : 0.f;
+        r4.y = gj + 1 < ncols ? rn_src[gj + 1] : 0.f;
+        r4.z = gj + 2 < ncols ? rn_src[gj + 2] : 0.f;
+        r4.w = gj + 3 < ncols ? rn_src[gj + 3] : 0.f;
       }
-      __syncwarp();
-      if (!__all_sync(0xffffffffu, mbar_wait(&sh.acc_full[a], (tcount >> 1) & 1))) { ok = false; break; }
-      tc_fence_after();
       const int row = tmi * BM + qd * 32 + lane;
       const bool row_ok = row < nrows;
       const bool kept_space = MODE == MODE_GRAM || kept_rows;
       const float rni = row_ok ? (kept_space ? im.rnk[row] : im.rn[row]) : 0.f;
-      const uint32_t taddr = tmem_base + a * BN + ((uint32_t)(qd * 32) << 16);
+      __syncwarp();
+      reinterpret_cast<float4 *>(rn_col)[lane] = r4;
+      __syncwarp();
+      if (!__all_sync(0xffffffffu, mbar_wait(&sh.acc_full[a], (tcount >> 1) & 1))) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + a * BN + half * HALF + ((uint32_t)(qd * 32) << 16);
       unsigned long long rowsum = 0ull;
-      unsigned long long best = kBestInit;
-#pragma unroll 1
-      for (int ch = 0; ch < BN / 32; ++ch) {
-        uint32_t v[32];
-        tmem_ld32(taddr + ch * 32, v);
+      float bd = 3.0f;                              // best distance so far (assignment); distances are <= 2
+      int bi = 0;
+      uint32_t v[2][32];
+      tmem_ld32(taddr, v[0]);
+#pragma unroll
+      for (int ch = 0; ch < HALF / 32; ++ch) {
         tmem_ld_wait();
-        const int c0 = tni * BN + ch * 32;
-        if (c0 >= ncols) continue;                  // uniform
-        if (MODE == MODE_GRAM) {
-          uint32_t bits = 0u;
-          unsigned long long s = 0ull;
-#pragma unroll
-          for (int k = 0; k < 32; ++k) {
-            const int gj = c0 + k;
-            float dd = DistF::dist(__uint_as_float(v[k]), rni, rn_col[ch * 32 + k]);
-            if (gj == row) dd = 0.f;
-            if (gj < ncols) {
-              s += DistF::term(dd, im);
-              if (DistF::within(dd, im)) bits |= 1u << k;
-              if (row < gj && DistF::in_band(dd, im)) ++band;
+        if (ch + 1 < HALF / 32) tmem_ld32(taddr + (ch + 1) * 32, v[(ch + 1) & 1]);
+        const int c0 = cbase + ch * 32;
+        if (c0 < ncols) {                           // uniform
+          const uint32_t(&vv)[32] = v[ch & 1];
+          const int r0 = tmi * BM + qd * 32;
+          if (MODE == MODE_GRAM) {
+            uint32_t bits;
+            const bool edge = (c0 + 32 > ncols) || (c0 < r0 + 32 && c0 + 32 > r0);
+            if (edge) gram_chunk<true>(vv, rn_col + ch * 32, rni, row, c0, ncols, im, rowsum, bits, band);
+            else {
+              int bnd = 0;
+              gram_chunk<false>(vv, rn_col + ch * 32, rni, row, c0, ncols, im, rowsum, bits, bnd);
+              if (row < c0) band += bnd;            // each unordered pair once; the chunk lies wholly on one side
             }
-          }
-          if (row_ok) {
-            rowsum += s;
-            im.adj[(size_t)row * im.Wp + (c0 >> 5)] = bits;
-          }
-        } else {
+            if (row_ok) im.adj[(size_t)row * im.Wp + (c0 >> 5)] = bits;
+          } else {
+            const int lim = min(32, ncols - c0);
 #pragma unroll
-          for (int k = 0; k < 32; ++k) {
-            const int gj = c0 + k;
-            const float dd = DistF::dist(__uint_as_float(v[k]), rni, rn_col[ch * 32 + k]);
-            const unsigned long long pk = ((unsigned long long)__float_as_uint(dd) << 32) | (unsigned)gj;
-            if (gj < ncols && pk < best) best = pk;
+            for (int k4 = 0; k4 < 32; k4 += 4) {
+              const float4 rn4 = *reinterpret_cast<const float4 *>(rn_col + ch * 32 + k4);
+              const float rnj[4] = {rn4.x, rn4.y, rn4.z, rn4.w};
+#pragma unroll
+              for (int kk = 0; kk < 4; ++kk) {
+                const int k = k4 + kk;
+                const float dd = DistF::dist(__uint_as_float(vv[k]), rni, rnj[kk]);
+                if (k < lim && dd < bd) { bd = dd; bi = c0 + k; }
+              }
+            }
           }
         }
       }
-      // the accumulator may be overwritten once all four epilogue warps have read it
+      // the accumulator may be overwritten once all epilogue warps have read it
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh.acc_empty[a]);
       if (row_ok) {
         if (MODE == MODE_GRAM) atomicAdd(&im.rho_fix[row], rowsum);
-        else atomicMin(&im.best[kept_rows ? im.kept_idx[row] : row], best);
+        else if (bd <= 2.0f) {
+          const unsigned long long pk = ((unsigned long long)__float_as_uint(bd) << 32) | (unsigned)bi;
+          atomicMin(&im.best[kept_rows ? im.kept_idx[row] : row], pk);
+        }
       }
     }
     if (!ok) atomicExch(&sh.abort, 1);
@@ -347,7 +402,7 @@ cudaError_t launch_gram_umma(const Batch &bt, int maxN, const ClusterCfg &cfg, c
     tm.b[b] = tm.a[b];
   }
   dim3 grid(umma_grid_x(maxN, maxN, bt.B, cfg.sm_count), bt.B);
-  k_tiles_umma<MODE_GRAM><<<grid, 192, kUmmaSmem, st>>>(bt, tm, 0);
+  k_tiles_umma<MODE_GRAM><<<grid, THREADS, kUmmaSmem, st>>>(bt, tm, 0);
   return cudaGetLastError();
 }
 
@@ -361,7 +416,7 @@ cudaError_t launch_assign_umma(const Batch &bt, int maxN, bool kept_rows, const 
     if (!encode_rows(&tm.b[b], im.Kcen, im.Np, bt.d_k, bt.d_k)) return cudaErrorInvalidValue;
   }
   dim3 grid(umma_grid_x(maxN, maxN, bt.B, cfg.sm_count), bt.B);
-  k_tiles_umma<MODE_ASSIGN><<<grid, 192, kUmmaSmem, st>>>(bt, tm, kept_rows ? 1 : 0);
+  k_tiles_umma<MODE_ASSIGN><<<grid, THREADS, kUmmaSmem, st>>>(bt, tm, kept_rows ? 1 : 0);
   return cudaGetLastError();
 }
 
