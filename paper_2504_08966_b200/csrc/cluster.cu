@@ -204,27 +204,49 @@ __global__ void __launch_bounds__(256) k_gram_simt(const __grid_constant__ Batch
 }
 
 // ---- density rank: rank_i = #{ j : rho_j > rho_i, or rho_j == rho_i and j < i } ------------------
-// grid (n_ctas, B) persistent over 256 x 256 blocks of pairs.
+// grid (n_ctas, B) persistent over 256 x 256 blocks of pairs.  The loop compares the upper 32 of
+// the 48 significant bits of the integer densities; a row that meets an equal upper word anywhere in
+// the block (rare) repeats the block with full comparisons.
+constexpr int kRankShift = 16;
 __global__ void __launch_bounds__(256) k_rank(const __grid_constant__ Batch bt) {
   const ImgDesc &im = bt.img[blockIdx.y];
   const int q = *im.q_ptr;
   const int nb = (q + 255) / 256;
   const int t = threadIdx.x;
+  __shared__ __align__(16) uint32_t khi[256];
   __shared__ unsigned long long keys[256];
   for (int blk = blockIdx.x; blk < nb * nb; blk += gridDim.x) {
     const int bi = blk / nb, bj = blk % nb;
     const int j0 = bj * 256;
-    __syncthreads();
-    keys[t] = (j0 + t < q) ? im.rho_fix[j0 + t] : 0ull;
-    __syncthreads();
     const int i = bi * 256 + t;
+    const unsigned long long mine = i < q ? im.rho_fix[i] : 0ull;
+    const unsigned long long other = (j0 + t < q) ? im.rho_fix[j0 + t] : 0ull;
+    __syncthreads();
+    keys[t] = other;
+    // rows past the end get an upper word of 0 and can only tie with a density of zero; the tie
+    // path below sorts that out by index
+    khi[t] = (uint32_t)(other >> kRankShift);
+    __syncthreads();
     if (i < q) {
-      const unsigned long long mine = im.rho_fix[i];
+      const uint32_t mh = (uint32_t)(mine >> kRankShift);
       const int nj = min(256, q - j0);
-      int c = 0;
-      for (int j = 0; j < nj; ++j) {
-        const unsigned long long o = keys[j];
-        c += (o > mine) || (o == mine && (j0 + j) < i);
+      int c = 0, eq = 0;
+      if (nj == 256) {
+#pragma unroll 4
+        for (int j = 0; j < 256; j += 4) {
+          const uint4 o = *reinterpret_cast<const uint4 *>(&khi[j]);
+          c += (o.x > mh) + (o.y > mh) + (o.z > mh) + (o.w > mh);
+          eq += (o.x == mh) + (o.y == mh) + (o.z == mh) + (o.w == mh);
+        }
+      } else {
+        for (int j = 0; j < nj; ++j) { c += khi[j] > mh; eq += khi[j] == mh; }
+      }
+      if (eq > (bi == bj ? 1 : 0)) {              // the row itself always ties in a diagonal block
+        c = 0;
+        for (int j = 0; j < nj; ++j) {
+          const unsigned long long o = keys[j];
+          c += (o > mine) || (o == mine && (j0 + j) < i);
+        }
       }
       if (c) atomicAdd(&im.rank[i], c);
       if (bj == 0) {
@@ -507,7 +529,7 @@ void launch_gram(const Batch &bt, int maxN, bool bf16, const ClusterCfg &cfg, cu
 
 void launch_rank(const Batch &bt, int maxN, const ClusterCfg &cfg, cudaStream_t st) {
   const long long nb = (maxN + 255) / 256;
-  dim3 grid(tile_grid(nb * nb, cfg.sm_count * 8), bt.B);
+  dim3 grid(tile_grid(nb * nb, cfg.sm_count * 4), bt.B);
   k_rank<<<grid, 256, 0, st>>>(bt);
 }
 

@@ -156,31 +156,34 @@ __global__ void __launch_bounds__(1024) k_logits(const __grid_constant__ Batch b
     for (int u = 0; u < UK; ++u)
       if (lane + 32 * u < nv) kb[u] = __ldg(krow + lane + 32 * u);
   }
-  for (int c = t; c < bt.n_qcols; c += 1024) qg[c] = im.qg[c];
+  // the global query is kept transposed, qT[k][vq] = Qglobal[vq * V + k], so that the lanes of a warp,
+  // which hold consecutive 16-byte vectors of the key row, read consecutive doubles
+  const int nvq = bt.n_qcols / V;
+  for (int c = t; c < bt.n_qcols; c += 1024) qg[(c % V) * nvq + c / V] = im.qg[c];
   __syncthreads();
   if (r < r1) {
+    const int vph = d_h / V;                                  // vectors per head
     for (int j = 0; j < n_qh; ++j) {
       double acc = 0.0;
       if (use_query) {
         const int kv = (j * bt.n_kvh) / n_qh;
-        const double *qr = qg + (size_t)j * d_h - (size_t)kv * d_h;    // indexed by the element's place in the row
+        const int vshift = (j - kv) * vph;                    // key-row vector v pairs with query vector v + vshift
 #pragma unroll
         for (int u = 0; u < UK; ++u) {
-          const int e0 = (lane + 32 * u) * V;
-          if (lane + 32 * u < nv && e0 / d_h == kv) {
+          const int v = lane + 32 * u;
+          if (v < nv && v / vph == kv) {
             float x[V];
             widen_vec<T>(kb[u], x);
 #pragma unroll
-            for (int k = 0; k < V; ++k) acc = fma((double)x[k], qr[e0 + k], acc);
+            for (int k = 0; k < V; ++k) acc = fma((double)x[k], qg[k * nvq + v + vshift], acc);
           }
         }
-        for (int v = lane + 32 * UK; v < nv; v += 32) {               // rows wider than the preloaded part
-          const int e0 = v * V;
-          if (e0 / d_h == kv) {
+        for (int v = lane + 32 * UK; v < nv; v += 32) {       // rows wider than the preloaded part
+          if (v / vph == kv) {
             float x[V];
             widen_vec<T>(__ldg(krow + v), x);
 #pragma unroll
-            for (int k = 0; k < V; ++k) acc = fma((double)x[k], qr[e0 + k], acc);
+            for (int k = 0; k < V; ++k) acc = fma((double)x[k], qg[k * nvq + v + vshift], acc);
           }
         }
         acc = warp_sum(acc);
@@ -284,6 +287,7 @@ __global__ void __launch_bounds__(1024) k_select_gather(const __grid_constant__ 
   int *own = reinterpret_cast<int *>(dsm + (keys_in_smem ? N : 0));   // [own_cap]
   __shared__ int hist[256];
   __shared__ int warp_tot[32];
+  __shared__ uint32_t wmin[32], wmax[32];
   __shared__ uint32_t s_prefix;
   __shared__ int s_k;
 
@@ -295,26 +299,40 @@ __global__ void __launch_bounds__(1024) k_select_gather(const __grid_constant__ 
     for (int wd = gt; wd < im.Wp; wd += gs) { im.cmask[wd] = 0u; im.rmask[wd] = 0u; }
     for (int i = gt; i < N; i += gs) im.best[i] = kBestInit;
   }
-  if (t == 0) { s_prefix = 0; s_k = im.m_target; }
+  if (t == 0) s_k = im.m_target;
   if (t < 256) hist[t] = 0;
   __syncthreads();
   auto key = [&](int i) -> uint32_t { return keys_in_smem ? skey[i] : score_key(im.score[i]); };
 
-  // radix select of the (m_target + 1)-th smallest key, most significant byte first; lanes of a
-  // warp that hit the same bin add once
-  uint32_t mask = 0;
+  // The bits above the highest bit in which two keys differ are common to all keys and need no pass.
   const int rounds = (N + 1023) / 1024;
-  for (int pass = 3; pass >= 0; --pass) {
-    const int shift = pass * 8;
+  uint32_t kmin = 0xffffffffu, kmax = 0u;
+  for (int it = 0; it < rounds; ++it) {
+    const int i = it * 1024 + t;
+    if (i < N) { const uint32_t kk = key(i); kmin = min(kmin, kk); kmax = max(kmax, kk); }
+  }
+  kmin = __reduce_min_sync(0xffffffffu, kmin);
+  kmax = __reduce_max_sync(0xffffffffu, kmax);
+  if (lane == 0) { wmin[w] = kmin; wmax[w] = kmax; }
+  __syncthreads();
+  kmin = __reduce_min_sync(0xffffffffu, wmin[lane]);
+  kmax = __reduce_max_sync(0xffffffffu, wmax[lane]);
+  const int top = 32 - __clz(kmin ^ kmax);                  // low bits that vary (0: all keys are equal)
+  if (t == 0) s_prefix = top >= 32 ? 0u : (kmin >> top) << top;
+  __syncthreads();
+
+  // radix select of the (m_target + 1)-th smallest key over the varying bits, up to 8 bits per pass
+  for (int hi = top; hi > 0; hi -= 8) {
+    const int lo = hi > 8 ? hi - 8 : 0;
+    const uint32_t dmask = (1u << (hi - lo)) - 1u;
+    const uint32_t above = hi >= 32 ? 0u : ~((1u << hi) - 1u);   // bits already fixed
     const uint32_t prefix = s_prefix;
     for (int it = 0; it < rounds; ++it) {
       const int i = it * 1024 + t;
-      bool valid = i < N;
-      uint32_t kk = 0;
-      if (valid) { kk = key(i); valid = (kk & mask) == prefix; }
-      const uint32_t dgt = (kk >> shift) & 255u;
-      const unsigned peers = __match_any_sync(0xffffffffu, valid ? dgt : (256u + lane));
-      if (valid && lane == __ffs(peers) - 1) atomicAdd(&hist[dgt], __popc(peers));
+      if (i < N) {
+        const uint32_t kk = key(i);
+        if ((kk & above) == (prefix & above)) atomicAdd(&hist[(kk >> lo) & dmask], 1);
+      }
     }
     __syncthreads();
     if (w == 0) {
@@ -341,12 +359,11 @@ __global__ void __launch_bounds__(1024) k_select_gather(const __grid_constant__ 
           }
         }
         s_k = kk;
-        s_prefix = prefix | ((uint32_t)(lane * 8 + dgt) << shift);
+        s_prefix = prefix | ((uint32_t)(lane * 8 + dgt) << lo);
       }
 #pragma unroll
       for (int b = 0; b < 8; ++b) hist[lane * 8 + b] = 0;
     }
-    mask |= 255u << shift;
     __syncthreads();
   }
   const uint32_t tau_key = s_prefix;
