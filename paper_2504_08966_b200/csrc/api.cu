@@ -9,7 +9,7 @@
 
 using namespace pact;
 
-constexpr int kProfStages = 12;
+constexpr int kProfStages = 10;
 
 struct pact_ctx {
   int d, n_qh, n_kvh, d_h, d_k, n_qcols;
@@ -32,8 +32,8 @@ struct pact_graph {
 };
 
 static const char *const kStageNames[kProfStages] = {
-    "prepass", "logits", "scores", "select_gather", "gram_density", "rank",
-    "centers", "centers_finalize", "assign", "label", "lists", "merge"};
+    "prepass", "logits", "scores", "select_gather", "gram_density", "centers", "assign", "label", "lists",
+    "merge"};
 
 namespace {
 
@@ -78,7 +78,6 @@ size_t carve_image(const pact_ctx *c, int N, char *base, ImgDesc *im) {
   cv.take(m.rho_fix, (size_t)Np * sizeof(unsigned long long));
   cv.take(m.rho, (size_t)Np * sizeof(float));
   cv.take(m.adj, (size_t)Np * Wp * sizeof(uint32_t));
-  cv.take(m.rank, (size_t)Np * sizeof(int32_t));
   cv.take(m.cmask, (size_t)Wp * sizeof(uint32_t));
   cv.take(m.rmask, (size_t)Wp * sizeof(uint32_t));
   cv.take(m.Kcen, (size_t)Np * c->d_k * c->elt);
@@ -365,13 +364,11 @@ pact_status pact_dbdpc(pact_ctx *ctx, const void *K, int64_t ldK, int N, const i
   launch_keynorm_gather(bt, N, bf, false, st);
   if (ctx->umma) CK(launch_gram_umma(bt, N, ctx->ccfg, st));
   else launch_gram(bt, N, bf, ctx->ccfg, st);
-  launch_rank(bt, N, ctx->ccfg, st);
-  CK(launch_centers(bt, ctx->ccfg, st));
-  launch_centers_finalize(bt, N, bf, ctx->ccfg, st);
+  CK(launch_centers(bt, N, bf, ctx->ccfg, st));
   if (ctx->umma) CK(launch_assign_umma(bt, N, true, ctx->ccfg, st));
   else launch_assign(bt, N, bf, ROWS_KEPT_LIST, ctx->ccfg, st);
   launch_label(bt, N, bf, ROWS_KEPT_LIST, st);
-  ctx->launches += 7;
+  ctx->launches += 5;
   CK(cudaGetLastError());
   if (counters)
     CK(cudaMemcpyAsync(counters, m.cnt, PACT_N_COUNTERS * sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
@@ -467,7 +464,7 @@ pact_status pact_reduce(pact_ctx *ctx, const pact_image *imgs, int B, const pact
     Batch bt;
     memset(&bt, 0, sizeof(bt));
     set_dims(ctx, bt, nb);
-    int cmaxN = 0;
+    int cmaxN = 0, cmaxQ = 0;
     for (int b = 0; b < nb; ++b) {
       ImgDesc &m = bt.img[b];
       const pact_image *g = imgs + b0 + b;
@@ -476,6 +473,8 @@ pact_status pact_reduce(pact_ctx *ctx, const pact_image *imgs, int B, const pact
       set_params(m, params + (size_t)(b0 + b) * params_stride, g->N);
       point_counts_at_workspace(m);
       cmaxN = g->N > cmaxN ? g->N : cmaxN;
+      const int qest = g->N - m.m_target + 64 < g->N ? g->N - m.m_target + 64 : g->N;   // survivors, with room for ties
+      cmaxQ = qest > cmaxQ ? qest : cmaxQ;
       CK(cudaMemsetAsync(m.cnt, 0, 32 * sizeof(int32_t), st));
     }
     int stage = 0;
@@ -493,16 +492,14 @@ pact_status pact_reduce(pact_ctx *ctx, const pact_image *imgs, int B, const pact
     if (ctx->umma) CK(launch_gram_umma(bt, cmaxN, ctx->ccfg, st));
     else launch_gram(bt, cmaxN, bf, ctx->ccfg, st);
     CK(mark());
-    launch_rank(bt, cmaxN, ctx->ccfg, st);          CK(mark());
-    CK(launch_centers(bt, ctx->ccfg, st));          CK(mark());
-    launch_centers_finalize(bt, cmaxN, bf, ctx->ccfg, st);  CK(mark());
+    CK(launch_centers(bt, cmaxQ, bf, ctx->ccfg, st));  CK(mark());
     if (ctx->umma) CK(launch_assign_umma(bt, cmaxN, false, ctx->ccfg, st));
     else launch_assign(bt, cmaxN, bf, ROWS_ALL, ctx->ccfg, st);
     CK(mark());
     launch_label(bt, cmaxN, bf, ROWS_ALL, st);      CK(mark());
     launch_lists(bt, cmaxN, st);                    CK(mark());
     launch_merge(bt, cmaxN, bf, ctx->out == PACT_BF16, ctx->ccfg, st);  CK(mark());
-    ctx->launches += 12;
+    ctx->launches += 10;
     CK(cudaGetLastError());
     for (int b = 0; b < nb; ++b)
       CK(cudaMemcpyAsync(bt.img[b].counters_user, bt.img[b].cnt, PACT_N_COUNTERS * sizeof(int32_t),

@@ -4,6 +4,8 @@
 //
 // This file holds the SIMT tile kernels (any element type and key width); the tcgen05 tile
 // kernels for bf16 keys live in gram_umma.cu and share the epilogue arithmetic of common.cuh.
+#include <cooperative_groups.h>
+
 #include "kernels.cuh"
 
 namespace pact {
@@ -30,7 +32,7 @@ __global__ void __launch_bounds__(256) k_keynorm_gather(const __grid_constant__ 
   // per-call initialisation of the arrays later kernels accumulate into
   {
     const int gt = blockIdx.x * 256 + threadIdx.x, gs = gridDim.x * 256;
-    for (int r = gt; r < im.Np; r += gs) { im.rho_fix[r] = 0ull; im.rank[r] = 0; }
+    for (int r = gt; r < im.Np; r += gs) im.rho_fix[r] = 0ull;
     for (int wd = gt; wd < im.Wp; wd += gs) { im.cmask[wd] = 0u; im.rmask[wd] = 0u; }
     for (int i = gt; i < im.N; i += gs) {
       im.best[i] = kBestInit;
@@ -203,71 +205,30 @@ __global__ void __launch_bounds__(256) k_gram_simt(const __grid_constant__ Batch
   if (band) atomicAdd(&im.cnt[PACT_CNT_BAND_DC], band);
 }
 
-// ---- density rank: rank_i = #{ j : rho_j > rho_i, or rho_j == rho_i and j < i } ------------------
-// grid (n_ctas, B) persistent over 256 x 256 blocks of pairs.  The loop compares the upper 32 of
-// the 48 significant bits of the integer densities; a row that meets an equal upper word anywhere in
-// the block (rare) repeats the block with full comparisons.
-constexpr int kRankShift = 16;
-__global__ void __launch_bounds__(256) k_rank(const __grid_constant__ Batch bt) {
-  const ImgDesc &im = bt.img[blockIdx.y];
-  const int q = *im.q_ptr;
-  const int nb = (q + 255) / 256;
-  const int t = threadIdx.x;
-  __shared__ __align__(16) uint32_t khi[256];
-  __shared__ unsigned long long keys[256];
-  for (int blk = blockIdx.x; blk < nb * nb; blk += gridDim.x) {
-    const int bi = blk / nb, bj = blk % nb;
-    const int j0 = bj * 256;
-    const int i = bi * 256 + t;
-    const unsigned long long mine = i < q ? im.rho_fix[i] : 0ull;
-    const unsigned long long other = (j0 + t < q) ? im.rho_fix[j0 + t] : 0ull;
-    __syncthreads();
-    keys[t] = other;
-    // rows past the end get an upper word of 0 and can only tie with a density of zero; the tie
-    // path below sorts that out by index
-    khi[t] = (uint32_t)(other >> kRankShift);
-    __syncthreads();
-    if (i < q) {
-      const uint32_t mh = (uint32_t)(mine >> kRankShift);
-      const int nj = min(256, q - j0);
-      int c = 0, eq = 0;
-      if (nj == 256) {
-#pragma unroll 4
-        for (int j = 0; j < 256; j += 4) {
-          const uint4 o = *reinterpret_cast<const uint4 *>(&khi[j]);
-          c += (o.x > mh) + (o.y > mh) + (o.z > mh) + (o.w > mh);
-          eq += (o.x == mh) + (o.y == mh) + (o.z == mh) + (o.w == mh);
-        }
-      } else {
-        for (int j = 0; j < nj; ++j) { c += khi[j] > mh; eq += khi[j] == mh; }
-      }
-      if (eq > (bi == bj ? 1 : 0)) {              // the row itself always ties in a diagonal block
-        c = 0;
-        for (int j = 0; j < nj; ++j) {
-          const unsigned long long o = keys[j];
-          c += (o > mine) || (o == mine && (j0 + j) < i);
-        }
-      }
-      if (c) atomicAdd(&im.rank[i], c);
-      if (bj == 0) {
-        const float rf = (float)((double)mine * (1.0 / (double)(1u << kRhoShift)));
-        im.rho[i] = rf;
-        if (im.rho_user) im.rho_user[i] = rf;
-      }
-    }
-  }
-}
-
 // ---- centre selection -------------------------------------------------------------------------
 // The sequential loop of Algorithm 2 picks the lexicographically first maximal independent set of
-// the graph {d_ij <= d_c} in density order; that set is unique, so any schedule that only takes
-// final decisions reproduces it (the argument of Appendix D.2).  A row becomes
-//   removed  once an earlier-ranked neighbour is a centre,
-//   a centre once every earlier-ranked neighbour is removed.
+// the graph {d_ij <= d_c} in density order (ties: lower index first); that set is unique, so any
+// schedule that only takes final decisions reproduces it (the argument of Appendix D.2).  A row becomes
+//   removed  once an earlier neighbour is a centre,
+//   a centre once every earlier neighbour is removed.
 // Both facts are monotone bits, so rows are resolved asynchronously: each warp owns rows, re-reads
-// the two bit masks and decides what it can, until all its rows are decided.  Launched
-// cooperatively so that every CTA is resident; every wait is bounded.
-__global__ void __launch_bounds__(256) k_centers(const __grid_constant__ Batch bt) {
+// the two bit masks and decides what it can, until all its rows are decided.
+//
+// One cooperative kernel (every CTA resident), 256 threads, three parts:
+//  1. "earlier" is decided from the integer densities themselves (no rank array): the densities of an
+//     image are staged in shared memory, each warp masks the adjacency words of its rows down to the
+//     earlier neighbours (written back, and the first row's words stay in registers);
+//  2. resolution loop (bounded);
+//  3. after a grid-wide barrier: cluster ids (number of centres with a lower index), centre list,
+//     centre keys and inverse norms.
+constexpr int kAdjRegs = 8;      // adjacency words per lane kept in registers: rows of up to 8192 survivors
+
+template <typename T>
+__global__ void __launch_bounds__(256) k_centers(const __grid_constant__ Batch bt, int keys_cap) {
+  using D = typename DistOf<T>::type;
+  constexpr int V = Vec<T>::N;
+  cooperative_groups::grid_group grid = cooperative_groups::this_grid();
+  extern __shared__ unsigned long long skeys[];          // [keys_cap] densities of the current image
   const int lane = threadIdx.x & 31;
   const int nwarps = gridDim.x * 8;
   const int gw = blockIdx.x * 8 + (threadIdx.x >> 5);
@@ -275,28 +236,68 @@ __global__ void __launch_bounds__(256) k_centers(const __grid_constant__ Batch b
   qs[0] = 0;
   for (int b = 0; b < bt.B; ++b) qs[b + 1] = qs[b] + *bt.img[b].q_ptr;
   const int total = qs[bt.B];
-  // phase 1: keep only the neighbours that come earlier in density order
-  for (int item = gw; item < total; item += nwarps) {
-    int b = 0;
-    while (item >= qs[b + 1]) ++b;
+
+  // part 1: keep only the neighbours that come earlier in density order
+  uint32_t cached[kAdjRegs];
+  int cached_item = -1;
+  for (int b = 0; b < bt.B; ++b) {
     const ImgDesc &im = bt.img[b];
-    const int r = item - qs[b], q = qs[b + 1] - qs[b], nw = (q + 31) >> 5;
-    const int myrank = im.rank[r];
-    uint32_t *row = im.adj + (size_t)r * im.Wp;
-    for (int wd = lane; wd < nw; wd += 32) {
-      uint32_t bits = row[wd], out = 0u;
-      while (bits) {
-        const int bpos = __ffs(bits) - 1;
-        bits &= bits - 1;
-        const int j = wd * 32 + bpos;
-        if (j != r && im.rank[j] < myrank) out |= 1u << bpos;
+    const int q = qs[b + 1] - qs[b], nw = (q + 31) >> 5;
+    const bool in_smem = q <= keys_cap;
+    __syncthreads();
+    if (in_smem)
+      for (int r = threadIdx.x; r < q; r += 256) skeys[r] = im.rho_fix[r];
+    __syncthreads();
+    const unsigned long long *keys = in_smem ? skeys : im.rho_fix;
+    // first item of this warp that lies in image b
+    int item = gw;
+    if (item < qs[b]) item += ((qs[b] - item + nwarps - 1) / nwarps) * nwarps;
+    for (; item < qs[b + 1]; item += nwarps) {
+      const int r = item - qs[b];
+      const unsigned long long mine = keys[r];
+      uint32_t *row = im.adj + (size_t)r * im.Wp;
+      const bool keep_regs = cached_item < 0 && nw <= 32 * kAdjRegs;
+      uint32_t w_in[kAdjRegs];
+#pragma unroll
+      for (int u = 0; u < kAdjRegs; ++u) w_in[u] = (lane + 32 * u < nw) ? row[lane + 32 * u] : 0u;
+#pragma unroll
+      for (int u = 0; u < kAdjRegs; ++u) {
+        const int wd = lane + 32 * u;
+        uint32_t bits = w_in[u], out = 0u;
+        while (bits) {
+          const int bpos = __ffs(bits) - 1;
+          bits &= bits - 1;
+          const int j = wd * 32 + bpos;
+          const unsigned long long o = keys[j];
+          if (j != r && (o > mine || (o == mine && j < r))) out |= 1u << bpos;
+        }
+        if (wd < nw) row[wd] = out;
+        if (keep_regs) cached[u] = out;
       }
-      row[wd] = out;
+      for (int wd = lane + 32 * kAdjRegs; wd < nw; wd += 32) {     // rows longer than the register part
+        uint32_t bits = row[wd], out = 0u;
+        while (bits) {
+          const int bpos = __ffs(bits) - 1;
+          bits &= bits - 1;
+          const int j = wd * 32 + bpos;
+          const unsigned long long o = keys[j];
+          if (j != r && (o > mine || (o == mine && j < r))) out |= 1u << bpos;
+        }
+        row[wd] = out;
+      }
+      if (keep_regs) cached_item = item;
+      if (lane == 0) {
+        const float rf = (float)((double)mine * (1.0 / (double)(1u << kRhoShift)));
+        im.rho[r] = rf;
+        if (im.rho_user) im.rho_user[r] = rf;
+      }
     }
   }
   __syncwarp();
-  // phase 2: resolve
+
+  // part 2: resolve
   int sweeps = 0, pending = 1;
+  bool cached_done = false;
   while (pending && sweeps < kSpinLimit) {
     pending = 0;
     ++sweeps;
@@ -306,23 +307,41 @@ __global__ void __launch_bounds__(256) k_centers(const __grid_constant__ Batch b
       const ImgDesc &im = bt.img[b];
       const int r = item - qs[b], q = qs[b + 1] - qs[b], nw = (q + 31) >> 5;
       const uint32_t mybit = 1u << (r & 31);
-      const uint32_t decided = (ld_relaxed_u32(&im.cmask[r >> 5]) | ld_relaxed_u32(&im.rmask[r >> 5])) & mybit;
-      if (decided) continue;
-      const uint32_t *row = im.adj + (size_t)r * im.Wp;
       bool hit_center = false, alive = false;
-      for (int wd = lane; wd < nw; wd += 32) {
-        const uint32_t e = row[wd];
-        if (e) {
-          hit_center |= (e & ld_relaxed_u32(&im.cmask[wd])) != 0u;
-          alive |= (e & ~ld_relaxed_u32(&im.rmask[wd])) != 0u;
+      if (item == cached_item) {                  // the masked adjacency of this row is in registers
+        if (cached_done) continue;
+        uint32_t cm[kAdjRegs], rm[kAdjRegs];
+#pragma unroll
+        for (int u = 0; u < kAdjRegs; ++u) {
+          const bool need = cached[u] != 0u;
+          cm[u] = need ? ld_relaxed_u32(&im.cmask[lane + 32 * u]) : 0u;
+          rm[u] = need ? ld_relaxed_u32(&im.rmask[lane + 32 * u]) : 0u;
+        }
+#pragma unroll
+        for (int u = 0; u < kAdjRegs; ++u) {
+          hit_center |= (cached[u] & cm[u]) != 0u;
+          alive |= (cached[u] & ~rm[u]) != 0u;
+        }
+      } else {
+        const uint32_t decided = (ld_relaxed_u32(&im.cmask[r >> 5]) | ld_relaxed_u32(&im.rmask[r >> 5])) & mybit;
+        if (decided) continue;
+        const uint32_t *row = im.adj + (size_t)r * im.Wp;
+        for (int wd = lane; wd < nw; wd += 32) {
+          const uint32_t e = row[wd];
+          if (e) {
+            hit_center |= (e & ld_relaxed_u32(&im.cmask[wd])) != 0u;
+            alive |= (e & ~ld_relaxed_u32(&im.rmask[wd])) != 0u;
+          }
         }
       }
       hit_center = __any_sync(0xffffffffu, hit_center);
       alive = __any_sync(0xffffffffu, alive);
       if (hit_center) {
         if (lane == 0) atomicOr(&im.rmask[r >> 5], mybit);
+        if (item == cached_item) cached_done = true;
       } else if (!alive) {
         if (lane == 0) atomicOr(&im.cmask[r >> 5], mybit);
+        if (item == cached_item) cached_done = true;
       } else {
         pending = 1;
       }
@@ -334,61 +353,56 @@ __global__ void __launch_bounds__(256) k_centers(const __grid_constant__ Batch b
       atomicMax(&bt.img[b].cnt[PACT_CNT_SWEEPS], sweeps);
     }
   }
-}
 
-// ---- cluster ids, centre list, centre keys ------------------------------------------------------
-// grid (n_ctas, B), 256 threads; cluster id of a centre = number of centres with a lower index.
-template <typename T>
-__global__ void __launch_bounds__(256) k_centers_finalize(const __grid_constant__ Batch bt) {
-  using D = typename DistOf<T>::type;
-  constexpr int V = Vec<T>::N;
-  const ImgDesc &im = bt.img[blockIdx.y];
-  const int q = *im.q_ptr, nw = (q + 31) >> 5;
-  const int t = threadIdx.x, lane = t & 31, w = t >> 5;
-  extern __shared__ int pref[];            // [nw + 1] exclusive prefix of popcounts
-  __shared__ int wsum[8];
-  __shared__ int carry;
-  if (t == 0) carry = 0;
-  __syncthreads();
-  for (int base = 0; base < nw; base += 256) {
-    const int wd = base + t;
-    const int pc = wd < nw ? __popc(im.cmask[wd]) : 0;
-    int x = pc;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      int y = __shfl_up_sync(0xffffffffu, x, o);
-      if (lane >= o) x += y;
+  // part 3: every decision is final once all CTAs are here
+  __threadfence();
+  grid.sync();
+  for (int item = gw; item < total; item += nwarps) {
+    int b = 0;
+    while (item >= qs[b + 1]) ++b;
+    const ImgDesc &im = bt.img[b];
+    const int r = item - qs[b], q = qs[b + 1] - qs[b], nw = (q + 31) >> 5;
+    // this lane's words of the centre mask, its share of the row and the row's bookkeeping: one round trip
+    int below = 0, all = 0;
+    uint32_t myword = 0u;
+    for (int wd = lane; wd < nw; wd += 32) {
+      const uint32_t m = __ldcg(&im.cmask[wd]);
+      const int pc = __popc(m);
+      all += pc;
+      if (wd < (r >> 5)) below += pc;
+      else if (wd == (r >> 5)) { below += __popc(m & ((1u << (r & 31)) - 1u)); myword = m; }
     }
-    if (lane == 31) wsum[w] = x;
-    __syncthreads();
-    int off = carry;
-    for (int k = 0; k < w; ++k) off += wsum[k];
-    if (wd < nw) pref[wd] = off + x - pc;
-    __syncthreads();
-    if (t == 255) carry = off + x;
-    __syncthreads();
-  }
-  const int C = carry;
-  if (blockIdx.x == 0 && t == 0) {
-    im.cnt[PACT_CNT_C] = C;
-    if (im.C_user) *im.C_user = C;
-  }
-  const T *Kp = reinterpret_cast<const T *>(im.Kp);
-  T *Kcen = reinterpret_cast<T *>(im.Kcen);
-  for (int r = blockIdx.x * 8 + w; r < q; r += gridDim.x * 8) {
-    const uint32_t m = im.cmask[r >> 5];
-    if (!((m >> (r & 31)) & 1u)) continue;
-    const int c = pref[r >> 5] + __popc(m & ((1u << (r & 31)) - 1u));
+    const T *src = reinterpret_cast<const T *>(im.Kp) + (size_t)r * bt.d_k;
+    const int nv = bt.d_k / V;
+    uint4 buf[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (lane + 32 * u < nv) buf[u] = __ldcg(reinterpret_cast<const uint4 *>(src) + lane + 32 * u);
+    const int tok = im.kept_idx[r];
+    const auto rnr = rn_kept<D>(im)[r];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      below += __shfl_xor_sync(0xffffffffu, below, o);
+      all += __shfl_xor_sync(0xffffffffu, all, o);
+      myword |= __shfl_xor_sync(0xffffffffu, myword, o);
+    }
+    if (r == 0 && lane == 0) {
+      im.cnt[PACT_CNT_C] = all;
+      if (im.C_user) *im.C_user = all;
+    }
+    if (!((myword >> (r & 31)) & 1u)) continue;
+    const int c = below;
     if (lane == 0) {
       im.cid[r] = c;
-      const int tok = im.kept_idx[r];
       im.center_idx[c] = tok;
       if (im.center_idx_user) im.center_idx_user[c] = tok;
-      rn_cen<D>(im)[c] = rn_kept<D>(im)[r];
+      rn_cen<D>(im)[c] = rnr;
     }
-    for (int v = lane; v * V < bt.d_k; v += 32)
-      reinterpret_cast<uint4 *>(Kcen + (size_t)c * bt.d_k)[v] =
-          reinterpret_cast<const uint4 *>(Kp + (size_t)r * bt.d_k)[v];
+    uint4 *dst = reinterpret_cast<uint4 *>(reinterpret_cast<T *>(im.Kcen) + (size_t)c * bt.d_k);
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (lane + 32 * u < nv) dst[lane + 32 * u] = buf[u];
+    for (int v = lane + 128; v < nv; v += 32) dst[v] = __ldcg(reinterpret_cast<const uint4 *>(src) + v);
   }
 }
 
@@ -491,16 +505,18 @@ __global__ void __launch_bounds__(256) k_label(const __grid_constant__ Batch bt,
 // ---- launchers ---------------------------------------------------------------------------------
 
 cudaError_t cluster_configure(ClusterCfg *cfg) {
-  int dev = 0, sms = 0, per_sm = 0;
+  int dev = 0, sms = 0, optin = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return e;
-  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_centers, 256, 0);
+  e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
   if (e != cudaSuccess) return e;
   cfg->sm_count = sms;
-  cfg->centers_grid = sms * (per_sm < 1 ? 1 : (per_sm > 4 ? 4 : per_sm));
-  return cudaSuccess;
+  cfg->centers_smem_max = optin - 1024;
+  e = cudaFuncSetAttribute(k_centers<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, cfg->centers_smem_max);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(k_centers<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, cfg->centers_smem_max);
 }
 
 #define PACT_DISPATCH(bf16, KERNEL, ...)                       \
@@ -527,23 +543,22 @@ void launch_gram(const Batch &bt, int maxN, bool bf16, const ClusterCfg &cfg, cu
   PACT_DISPATCH(bf16, k_gram_simt, <<<grid, 256, 0, st>>>(bt));
 }
 
-void launch_rank(const Batch &bt, int maxN, const ClusterCfg &cfg, cudaStream_t st) {
-  const long long nb = (maxN + 255) / 256;
-  dim3 grid(tile_grid(nb * nb, cfg.sm_count * 4), bt.B);
-  k_rank<<<grid, 256, 0, st>>>(bt);
-}
-
-cudaError_t launch_centers(const Batch &bt, const ClusterCfg &cfg, cudaStream_t st) {
-  void *args[] = {(void *)&bt};
-  return cudaLaunchCooperativeKernel((const void *)k_centers, dim3(cfg.centers_grid), dim3(256), args, 0, st);
-}
-
-void launch_centers_finalize(const Batch &bt, int maxN, bool bf16, const ClusterCfg &cfg, cudaStream_t st) {
-  int maxWp = 0;
-  for (int b = 0; b < bt.B; ++b) maxWp = bt.img[b].Wp > maxWp ? bt.img[b].Wp : maxWp;
-  dim3 grid(tile_grid((maxN + 7) / 8, cfg.sm_count * 2), bt.B);
-  const size_t sm = (size_t)(maxWp + 1) * sizeof(int);
-  PACT_DISPATCH(bf16, k_centers_finalize, <<<grid, 256, sm, st>>>(bt));
+cudaError_t launch_centers(const Batch &bt, int maxQ, bool bf16, const ClusterCfg &cfg, cudaStream_t st) {
+  // the densities of one image are staged in shared memory when they fit in a quarter of it; maxQ is
+  // an estimate of the largest survivor count, an image with more reads them from global memory
+  size_t smem = (size_t)maxQ * sizeof(unsigned long long);
+  const size_t budget = (size_t)cfg.centers_smem_max / 4;
+  if (smem > budget) smem = 0;
+  int keys_cap = (int)(smem / sizeof(unsigned long long));
+  const void *fn = bf16 ? (const void *)k_centers<__nv_bfloat16> : (const void *)k_centers<float>;
+  int per_sm = 0;
+  cudaError_t e = bf16 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_centers<__nv_bfloat16>, 256, smem)
+                       : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_centers<float>, 256, smem);
+  if (e != cudaSuccess) return e;
+  if (per_sm < 1) return cudaErrorLaunchOutOfResources;
+  if (per_sm > 4) per_sm = 4;
+  void *args[] = {(void *)&bt, (void *)&keys_cap};
+  return cudaLaunchCooperativeKernel(fn, dim3(cfg.sm_count * per_sm), dim3(256), args, smem, st);
 }
 
 void launch_assign(const Batch &bt, int maxN, bool bf16, RowMode mode, const ClusterCfg &cfg, cudaStream_t st) {

@@ -49,7 +49,6 @@ struct ImgDesc {
   unsigned long long *rho_fix;  // [Np] integer density
   float *rho;            // [Np]
   uint32_t *adj;         // [Np][Wp] adjacency bits (d <= d_c), later masked to earlier neighbours
-  int32_t *rank;         // [Np]
   uint32_t *cmask;       // [Wp] centres
   uint32_t *rmask;       // [Wp] removed (within d_c of an earlier centre)
   void *Kcen;            // [Np][d_k] centre keys in cluster-id order

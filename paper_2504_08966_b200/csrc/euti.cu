@@ -295,7 +295,7 @@ __global__ void __launch_bounds__(1024) k_select_gather(const __grid_constant__ 
     for (int i = t; i < N; i += 1024) skey[i] = score_key(im.score[i]);
   if (do_gather) {   // per-call initialisation, spread over the grid
     const int gt = blockIdx.x * 1024 + t, gs = gridDim.x * 1024;
-    for (int r = gt; r < im.Np; r += gs) { im.rho_fix[r] = 0ull; im.rank[r] = 0; im.csize[r] = 0; im.cticket[r] = 0; }
+    for (int r = gt; r < im.Np; r += gs) { im.rho_fix[r] = 0ull; im.csize[r] = 0; im.cticket[r] = 0; }
     for (int wd = gt; wd < im.Wp; wd += gs) { im.cmask[wd] = 0u; im.rmask[wd] = 0u; }
     for (int i = gt; i < N; i += gs) im.best[i] = kBestInit;
   }

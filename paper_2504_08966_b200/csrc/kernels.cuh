@@ -22,16 +22,16 @@ cudaError_t select_configure();            // what launch_select_gather needs, o
 // cluster.cu
 struct ClusterCfg {
   int sm_count;
-  int centers_grid;     // CTAs of the cooperative centre-selection kernel
+  int centers_smem_max; // most dynamic shared memory the centre-selection kernel may ask for
 };
 cudaError_t cluster_configure(ClusterCfg *cfg);
 // gathers survivor keys and inverse norms; all_tokens: also every token's inverse norm
 void launch_keynorm_gather(const Batch &bt, int maxN, bool bf16, bool all_tokens, cudaStream_t st);
 void launch_center_key_gather(const Batch &bt, int maxN, bool bf16, cudaStream_t st);
 void launch_gram(const Batch &bt, int maxN, bool bf16, const ClusterCfg &cfg, cudaStream_t st);
-void launch_rank(const Batch &bt, int maxN, const ClusterCfg &cfg, cudaStream_t st);
-cudaError_t launch_centers(const Batch &bt, const ClusterCfg &cfg, cudaStream_t st);
-void launch_centers_finalize(const Batch &bt, int maxN, bool bf16, const ClusterCfg &cfg, cudaStream_t st);
+// density order, centre selection, cluster ids and centre keys in one cooperative kernel
+// maxQ: estimate of the largest number of survivors of an image (sizes the staging buffer only)
+cudaError_t launch_centers(const Batch &bt, int maxQ, bool bf16, const ClusterCfg &cfg, cudaStream_t st);
 void launch_assign(const Batch &bt, int maxN, bool bf16, RowMode mode, const ClusterCfg &cfg, cudaStream_t st);
 void launch_label(const Batch &bt, int maxN, bool bf16, RowMode mode, cudaStream_t st);
 
