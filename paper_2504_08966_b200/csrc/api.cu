@@ -180,7 +180,14 @@ pact_status check_image(const pact_ctx *c, const pact_image *g, bool need_euti, 
   return PACT_OK;
 }
 
+#ifdef PACT_TIMELINE
+unsigned long long *g_timeline = nullptr;
+#endif
+
 void fill_user(ImgDesc &m, const pact_image *g) {
+#ifdef PACT_TIMELINE
+  m.tl = g_timeline;
+#endif
   m.H = g->H; m.Ke = g->K_euti; m.Q = g->Q_euti; m.Kc = g->K_clu;
   m.ldH = g->ldH; m.ldKe = g->ldKe; m.ldQ = g->ldQ; m.ldKc = g->ldKc; m.ldHo = g->ldHo;
   m.P = g->P; m.H_out = g->H_out; m.P_out = g->P_out; m.size_out = g->size_out;
@@ -192,6 +199,11 @@ void fill_user(ImgDesc &m, const pact_image *g) {
 }  // namespace
 
 extern "C" {
+
+#ifdef PACT_TIMELINE
+// instrumented build only: device buffer of 16 x 4096 x 2 timestamps (zeroed by the caller)
+void pact_debug_set_timeline(unsigned long long *buf) { g_timeline = buf; }
+#endif
 
 const char *pact_status_string(pact_status s) {
   switch (s) {

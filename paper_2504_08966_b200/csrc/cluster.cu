@@ -228,6 +228,7 @@ __global__ void __launch_bounds__(256) k_centers(const __grid_constant__ Batch b
   using D = typename DistOf<T>::type;
   constexpr int V = Vec<T>::N;
   cooperative_groups::grid_group grid = cooperative_groups::this_grid();
+  TL_SCOPE(bt.img[0], 5);
   extern __shared__ unsigned long long skeys[];          // [keys_cap] densities of the current image
   const int lane = threadIdx.x & 31;
   const int nwarps = gridDim.x * 8;
@@ -469,6 +470,7 @@ template <typename T>
 __global__ void __launch_bounds__(256) k_label(const __grid_constant__ Batch bt, int mode) {
   using D = typename DistOf<T>::type;
   const ImgDesc &im = bt.img[blockIdx.y];
+  TL_SCOPE(im, 7);
   const int nrows = mode == ROWS_ALL ? im.N : (mode == ROWS_KEPT_LIST ? *im.q_ptr : *im.m_ptr);
   int joined = 0, dropped = 0, band = 0;
   for (int g = blockIdx.x * 256 + threadIdx.x; g < nrows; g += gridDim.x * 256) {

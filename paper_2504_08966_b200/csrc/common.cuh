@@ -71,6 +71,7 @@ struct ImgDesc {
   const int32_t *cidx_ptr;  // token index of centre c (workspace or caller)
   float *rho_user;       // optional outputs of the stage calls
   int32_t *center_idx_user, *C_user, *r_user;
+  unsigned long long *tl; // timeline buffer of the instrumented build (PACT_TIMELINE), else unused
   int Np, Wp;            // padded survivor capacity and words per adjacency row
   int bstride;           // entries per row of bstart
 };
@@ -80,6 +81,33 @@ struct Batch {
   int B;
   int d, n_qh, n_kvh, d_h, d_k, n_qcols;
 };
+
+// ---- optional per-CTA timeline (instrumented build only; compiles to nothing otherwise) ----------
+#ifdef PACT_TIMELINE
+constexpr int kTlCtas = 4096;
+struct TlScope {
+  unsigned long long *slot;
+  __device__ __forceinline__ TlScope(const ImgDesc &im, int kid) {
+    const unsigned cta = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
+    slot = (im.tl && cta < kTlCtas) ? im.tl + ((size_t)kid * kTlCtas + cta) * 2 : nullptr;
+    if (slot && threadIdx.x == 0) {
+      unsigned long long t;
+      asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+      slot[0] = t;
+    }
+  }
+  __device__ __forceinline__ ~TlScope() {
+    if (slot && (threadIdx.x & 31) == 0) {
+      unsigned long long t;
+      asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+      atomicMax(slot + 1, t);
+    }
+  }
+};
+#define TL_SCOPE(im, kid) TlScope tl_scope_(im, kid)
+#else
+#define TL_SCOPE(im, kid)
+#endif
 
 // ---- element access ----------------------------------------------------------------------
 

@@ -37,6 +37,7 @@ __global__ void __launch_bounds__(kPreThreads) k_prepass(const __grid_constant__
   using rn_t = typename D::rn_t;
   constexpr int V = Vec<T>::N;
   const ImgDesc &im = bt.img[blockIdx.y];
+  TL_SCOPE(im, 0);
   const int t = threadIdx.x, lane = t & 31, w = t >> 5;
   if ((int)blockIdx.x >= GQ) {
     const int tok = ((int)blockIdx.x - GQ) * kTokWarps + w;
@@ -131,54 +132,65 @@ __global__ void __launch_bounds__(kPreThreads) k_prepass(const __grid_constant__
 }
 
 // ---- Eq. 2, first half: logits and CTA-local softmax pieces ---------------------------------------
-// grid (ceil(maxN / 32), B), 1024 threads, dynamic smem (n_qcols + 32 n_qh) doubles.  One warp per
-// token: the whole key row is loaded at once, then every head takes its part of it.
+// grid (ceil(maxN / 32), B), 256 threads, dynamic smem (n_qcols + 32 n_qh) doubles.  A CTA takes 32
+// tokens, a warp four of them: their key rows are loaded at once, then every head takes its part.
+constexpr int kLogitThreads = 256;
+constexpr int kLogitTpw = kRowsPerCta / (kLogitThreads / 32);   // tokens per warp
+
 template <typename T>
-__global__ void __launch_bounds__(1024) k_logits(const __grid_constant__ Batch bt) {
+__global__ void __launch_bounds__(kLogitThreads) k_logits(const __grid_constant__ Batch bt) {
   const ImgDesc &im = bt.img[blockIdx.y];
+  TL_SCOPE(im, 1);
   constexpr int V = Vec<T>::N;
-  constexpr int UK = 4;
+  constexpr int UK = 2;                   // preloaded 16-byte vectors per lane and token
   const int g = blockIdx.x, t = threadIdx.x, lane = t & 31, w = t >> 5;
   const int G = (im.N + kRowsPerCta - 1) / kRowsPerCta;
   if (g >= G) return;
   extern __shared__ double smd[];
-  double *qg = smd;                       // [n_qcols]
+  double *qg = smd;                       // [n_qcols], transposed (see below)
   double *lg = smd + bt.n_qcols;          // [32][n_qh]
   const int n_qh = bt.n_qh, d_h = bt.d_h;
   const int r0 = g * kRowsPerCta, r1 = min(im.N, r0 + kRowsPerCta);
   const bool use_query = !(im.flags & PACT_FLAG_NORM_ONLY);
-  const int r = r0 + w;
   const int nv = bt.d_k / V;
-  const uint4 *krow = reinterpret_cast<const uint4 *>(reinterpret_cast<const T *>(im.Ke) + (size_t)min(r, im.N - 1) * im.ldKe);
-  uint4 kb[UK];
+  const T *K = reinterpret_cast<const T *>(im.Ke);
+  uint4 kb[kLogitTpw][UK];
   if (use_query) {
 #pragma unroll
-    for (int u = 0; u < UK; ++u)
-      if (lane + 32 * u < nv) kb[u] = __ldg(krow + lane + 32 * u);
+    for (int i = 0; i < kLogitTpw; ++i) {
+      const uint4 *krow = reinterpret_cast<const uint4 *>(K + (size_t)min(r0 + w * kLogitTpw + i, im.N - 1) * im.ldKe);
+#pragma unroll
+      for (int u = 0; u < UK; ++u)
+        if (lane + 32 * u < nv) kb[i][u] = __ldg(krow + lane + 32 * u);
+    }
   }
   // the global query is kept transposed, qT[k][vq] = Qglobal[vq * V + k], so that the lanes of a warp,
   // which hold consecutive 16-byte vectors of the key row, read consecutive doubles
   const int nvq = bt.n_qcols / V;
-  for (int c = t; c < bt.n_qcols; c += 1024) qg[(c % V) * nvq + c / V] = im.qg[c];
+  for (int c = t; c < bt.n_qcols; c += kLogitThreads) qg[(c % V) * nvq + c / V] = im.qg[c];
   __syncthreads();
-  if (r < r1) {
-    const int vph = d_h / V;                                  // vectors per head
+  const int vph = d_h / V;                                  // vectors per head
+#pragma unroll
+  for (int i = 0; i < kLogitTpw; ++i) {
+    const int lr = w * kLogitTpw + i;                       // token within the CTA
+    if (r0 + lr >= r1) break;
+    const uint4 *krow = reinterpret_cast<const uint4 *>(K + (size_t)(r0 + lr) * im.ldKe);
     for (int j = 0; j < n_qh; ++j) {
       double acc = 0.0;
       if (use_query) {
         const int kv = (j * bt.n_kvh) / n_qh;
-        const int vshift = (j - kv) * vph;                    // key-row vector v pairs with query vector v + vshift
+        const int vshift = (j - kv) * vph;                  // key-row vector v pairs with query vector v + vshift
 #pragma unroll
         for (int u = 0; u < UK; ++u) {
           const int v = lane + 32 * u;
           if (v < nv && v / vph == kv) {
             float x[V];
-            widen_vec<T>(kb[u], x);
+            widen_vec<T>(kb[i][u], x);
 #pragma unroll
             for (int k = 0; k < V; ++k) acc = fma((double)x[k], qg[k * nvq + v + vshift], acc);
           }
         }
-        for (int v = lane + 32 * UK; v < nv; v += 32) {       // rows wider than the preloaded part
+        for (int v = lane + 32 * UK; v < nv; v += 32) {     // rows wider than the preloaded part
           if (v / vph == kv) {
             float x[V];
             widen_vec<T>(__ldg(krow + v), x);
@@ -188,12 +200,12 @@ __global__ void __launch_bounds__(1024) k_logits(const __grid_constant__ Batch b
         }
         acc = warp_sum(acc);
       }
-      if (lane == 0) lg[w * n_qh + j] = acc;
+      if (lane == 0) lg[lr * n_qh + j] = acc;
     }
   }
   __syncthreads();
   // per head: CTA max, exp, CTA sum; lane = token within the CTA
-  for (int j = w; j < n_qh; j += 32) {
+  for (int j = w; j < n_qh; j += kLogitThreads / 32) {
     const int rr = r0 + lane;
     const bool ok = rr < r1;
     const double l = ok ? lg[lane * n_qh + j] : -1.0e300;
@@ -214,6 +226,7 @@ __global__ void __launch_bounds__(1024) k_logits(const __grid_constant__ Batch b
 // grid (ceil(maxN / 256), B), 256 threads.  Every CTA merges all pieces itself, one warp per head.
 __global__ void __launch_bounds__(256) k_scores(const __grid_constant__ Batch bt) {
   const ImgDesc &im = bt.img[blockIdx.y];
+  TL_SCOPE(im, 2);
   const int t = threadIdx.x, lane = t & 31, w = t >> 5;
   const int N = im.N, n_qh = bt.n_qh;
   if ((int)blockIdx.x * 256 >= N) return;
@@ -280,6 +293,7 @@ __global__ void __launch_bounds__(1024) k_select_gather(const __grid_constant__ 
                                                         int keys_in_smem, int own_cap) {
   using D = typename DistOf<T>::type;
   const ImgDesc &im = bt.img[blockIdx.y];
+  TL_SCOPE(im, 3);
   const int t = threadIdx.x, lane = t & 31, w = t >> 5;
   const int N = im.N;
   extern __shared__ uint32_t dsm[];
@@ -462,8 +476,8 @@ void launch_prepass(const Batch &bt, int maxN, bool bf16, cudaStream_t st) {
 void launch_logits(const Batch &bt, int maxN, bool bf16, cudaStream_t st) {
   dim3 grid((maxN + kRowsPerCta - 1) / kRowsPerCta, bt.B);
   const size_t sm = (size_t)(bt.n_qcols + kRowsPerCta * bt.n_qh) * sizeof(double);
-  if (bf16) k_logits<__nv_bfloat16><<<grid, 1024, sm, st>>>(bt);
-  else k_logits<float><<<grid, 1024, sm, st>>>(bt);
+  if (bf16) k_logits<__nv_bfloat16><<<grid, kLogitThreads, sm, st>>>(bt);
+  else k_logits<float><<<grid, kLogitThreads, sm, st>>>(bt);
 }
 
 void launch_scores(const Batch &bt, int maxN, cudaStream_t st) {

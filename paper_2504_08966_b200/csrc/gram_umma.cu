@@ -135,40 +135,58 @@ struct Shared {
 
 enum { MODE_GRAM = 0, MODE_ASSIGN = 1 };
 
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 // One 32-column chunk of the epilogue of the all-pairs pass for one row (= one lane): distance
 // (Eq. 5), density term (Eq. 6) as an integer multiple of 2^-30, adjacency bit d <= d_c, band count.
-// SLOW adds the per-element checks that only edge chunks need (diagonal, columns past the end).
-template <bool SLOW>
+// EDGE adds the per-element checks that only edge chunks need (diagonal, columns past the end).
+// The arithmetic is that of DistF (common.cuh) written out so that four terms are summed in 32 bits.
+template <bool EDGE>
 __device__ __forceinline__ void gram_chunk(const uint32_t (&v)[32], const float *rn_col, float rni, int row, int c0,
-                                           int ncols, const ImgDesc &im, unsigned long long &rowsum, uint32_t &bits,
-                                           int &band) {
+                                           int ncols, float d_c, float neg_k, unsigned long long &rowsum,
+                                           uint32_t &bits, int &band) {
   uint32_t b = 0u;
   unsigned long long s = 0ull;
+  int bnd = 0;
 #pragma unroll
   for (int k4 = 0; k4 < 32; k4 += 4) {
     const float4 rn4 = *reinterpret_cast<const float4 *>(rn_col + k4);
     const float rnj[4] = {rn4.x, rn4.y, rn4.z, rn4.w};
+    uint32_t s4 = 0u;                               // four terms, each at most 2^30, fit in 32 bits
 #pragma unroll
     for (int kk = 0; kk < 4; ++kk) {
       const int k = k4 + kk;
       float dd = DistF::dist(__uint_as_float(v[k]), rni, rnj[kk]);
-      if (SLOW) {
+      bool ok = true;
+      if (EDGE) {
         const int gj = c0 + k;
         if (gj == row) dd = 0.f;
-        if (gj < ncols) {
-          s += DistF::term(dd, im);
-          if (DistF::within(dd, im)) b |= 1u << k;
-          if (row < gj && DistF::in_band(dd, im)) ++band;
+        ok = gj < ncols;
+      }
+      const uint32_t term = __float2uint_rn(ex2_approx(dd * neg_k) * (float)(1u << kRhoShift));
+      const bool within = dd <= d_c;
+      const bool inband = fabsf(dd - d_c) <= 1e-6f;
+      if (EDGE) {
+        if (ok) {
+          s4 += term;
+          if (within) b |= 1u << k;
+          if (inband && row < c0 + k) ++bnd;
         }
       } else {
-        s += DistF::term(dd, im);
-        if (DistF::within(dd, im)) b |= 1u << k;
-        if (DistF::in_band(dd, im)) ++band;
+        s4 += term;
+        if (within) b |= 1u << k;
+        if (inband) ++bnd;
       }
     }
+    s += s4;
   }
   rowsum += s;
   bits = b;
+  band += bnd;
 }
 
 }  // namespace
@@ -179,6 +197,7 @@ template <int MODE>
 __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant__ Batch bt,
                                                            const __grid_constant__ TmapSet tm, int kept_rows) {
   const ImgDesc &im = bt.img[blockIdx.y];
+  TL_SCOPE(im, MODE == MODE_GRAM ? 4 : 6);
   extern __shared__ uint8_t smem_raw[];
   __shared__ Shared sh;
   uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -290,38 +309,36 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
       unsigned long long rowsum = 0ull;
       float bd = 3.0f;                              // best distance so far (assignment); distances are <= 2
       int bi = 0;
-      uint32_t v[2][32];
-      tmem_ld32(taddr, v[0]);
-#pragma unroll
+      const float d_c = im.d_c, neg_k = -im.inv_dn_log2e;
+      const int r0 = tmi * BM + qd * 32;
+#pragma unroll 1
       for (int ch = 0; ch < HALF / 32; ++ch) {
-        tmem_ld_wait();
-        if (ch + 1 < HALF / 32) tmem_ld32(taddr + (ch + 1) * 32, v[(ch + 1) & 1]);
         const int c0 = cbase + ch * 32;
-        if (c0 < ncols) {                           // uniform
-          const uint32_t(&vv)[32] = v[ch & 1];
-          const int r0 = tmi * BM + qd * 32;
-          if (MODE == MODE_GRAM) {
-            uint32_t bits;
-            const bool edge = (c0 + 32 > ncols) || (c0 < r0 + 32 && c0 + 32 > r0);
-            if (edge) gram_chunk<true>(vv, rn_col + ch * 32, rni, row, c0, ncols, im, rowsum, bits, band);
-            else {
-              int bnd = 0;
-              gram_chunk<false>(vv, rn_col + ch * 32, rni, row, c0, ncols, im, rowsum, bits, bnd);
-              if (row < c0) band += bnd;            // each unordered pair once; the chunk lies wholly on one side
-            }
-            if (row_ok) im.adj[(size_t)row * im.Wp + (c0 >> 5)] = bits;
-          } else {
-            const int lim = min(32, ncols - c0);
+        if (c0 >= ncols) break;                      // uniform
+        uint32_t v[32];
+        tmem_ld32(taddr + ch * 32, v);
+        tmem_ld_wait();
+        if (MODE == MODE_GRAM) {
+          uint32_t bits;
+          const bool edge = (c0 + 32 > ncols) || (c0 < r0 + 32 && c0 + 32 > r0);
+          if (edge) gram_chunk<true>(v, rn_col + ch * 32, rni, row, c0, ncols, d_c, neg_k, rowsum, bits, band);
+          else {
+            int bnd = 0;
+            gram_chunk<false>(v, rn_col + ch * 32, rni, row, c0, ncols, d_c, neg_k, rowsum, bits, bnd);
+            if (row < c0) band += bnd;              // each unordered pair once; the chunk lies wholly on one side
+          }
+          if (row_ok) im.adj[(size_t)row * im.Wp + (c0 >> 5)] = bits;
+        } else {
+          const int lim = min(32, ncols - c0);
 #pragma unroll
-            for (int k4 = 0; k4 < 32; k4 += 4) {
-              const float4 rn4 = *reinterpret_cast<const float4 *>(rn_col + ch * 32 + k4);
-              const float rnj[4] = {rn4.x, rn4.y, rn4.z, rn4.w};
+          for (int k4 = 0; k4 < 32; k4 += 4) {
+            const float4 rn4 = *reinterpret_cast<const float4 *>(rn_col + ch * 32 + k4);
+            const float rnj[4] = {rn4.x, rn4.y, rn4.z, rn4.w};
 #pragma unroll
-              for (int kk = 0; kk < 4; ++kk) {
-                const int k = k4 + kk;
-                const float dd = DistF::dist(__uint_as_float(vv[k]), rni, rnj[kk]);
-                if (k < lim && dd < bd) { bd = dd; bi = c0 + k; }
-              }
+            for (int kk = 0; kk < 4; ++kk) {
+              const int k = k4 + kk;
+              const float dd = DistF::dist(__uint_as_float(v[k]), rni, rnj[kk]);
+              if (k < lim && dd < bd) { bd = dd; bi = c0 + k; }
             }
           }
         }

@@ -84,6 +84,7 @@ __device__ __forceinline__ float4 ld_cg_f4(const float *p) {
 // integer atomics; the last block to finish turns them into chunk offsets for the merge.
 __global__ void __launch_bounds__(kListBlock) k_lists(const __grid_constant__ Batch bt) {
   const ImgDesc &im = bt.img[blockIdx.y];
+  TL_SCOPE(im, 8);
   const int N = im.N;
   const int nblk = (N + kListBlock - 1) / kListBlock;
   const int b = blockIdx.x, t = threadIdx.x;
@@ -167,6 +168,7 @@ template <typename T, typename O, int VPT>
 __global__ void __launch_bounds__(kMergeThreads) k_merge(const __grid_constant__ Batch bt) {
   constexpr int R = (sizeof(T) == 2 ? 16 : 8) / VPT;    // member rows in flight per thread
   const ImgDesc &im = bt.img[blockIdx.z];
+  TL_SCOPE(im, 9);
   const int t = threadIdx.x, lane = t & 31, w = t >> 5;
   const int C = *im.C_ptr;
   const int n_text = im.n_total - im.N;
