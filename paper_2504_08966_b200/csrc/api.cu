@@ -92,7 +92,6 @@ size_t carve_image(const pact_ctx *c, int N, char *base, ImgDesc *im) {
   cv.take(m.blocklist, nblk * 256 * sizeof(int32_t));
   cv.take(m.bstart, nblk * (size_t)m.bstride * sizeof(uint16_t));
   cv.take(m.csize, (size_t)Np * sizeof(int32_t));
-  cv.take(m.cbase, (size_t)Np * sizeof(int32_t));
   cv.take(m.cticket, (size_t)Np * sizeof(int32_t));
   cv.take(m.mpart, ((size_t)N / 8 + 2) * c->d * sizeof(float));
   return cv.off;
@@ -171,6 +170,7 @@ pact_status check_image(const pact_ctx *c, const pact_image *g, bool need_euti, 
     if (!g->K_clu || !aligned16(g->K_clu) || !ld_ok(c, g->ldKc, c->d_k)) return PACT_ERR_INVALID_ARG;
   }
   if (need_out) {
+    if (g->N > merge_max_tokens(c->d, c->elt)) return PACT_ERR_UNSUPPORTED;
     if (!g->H || !aligned16(g->H) || !ld_ok(c, g->ldH, c->d) || !g->P) return PACT_ERR_INVALID_ARG;
     if (!g->H_out || !aligned16(g->H_out) || !g->P_out || !g->size_out || !g->counters)
       return PACT_ERR_INVALID_ARG;
@@ -240,8 +240,9 @@ pact_status pact_create(pact_ctx **out, int d, int n_qh, int n_kvh, int d_h, pac
     e = cudaGetDeviceProperties(&pr, c->device);
     if (e == cudaSuccess && pr.major != 10) { delete c; return PACT_ERR_UNSUPPORTED; }
   }
-  if (e == cudaSuccess) e = euti_configure(c->n_qcols, c->n_qh);
+  if (e == cudaSuccess) e = euti_configure(c->n_qcols, c->n_qh, c->d, c->d_k, c->elt);
   if (e == cudaSuccess) e = cluster_configure(&c->ccfg);
+  if (e == cudaSuccess) e = merge_configure();
   if (e == cudaSuccess && in == PACT_BF16) e = umma_configure();
   if (e != cudaSuccess) {
     pact_status s = fail_cuda(ctx, e, "pact_create");
@@ -447,7 +448,7 @@ pact_status pact_merge(pact_ctx *ctx, const pact_image *img, const int32_t *labe
   CK(cudaMemsetAsync(m.csize, 0, (size_t)m.Np * sizeof(int32_t), st));
   CK(cudaMemsetAsync(m.cticket, 0, (size_t)m.Np * sizeof(int32_t), st));
   launch_lists(bt, img->N, st);
-  launch_merge(bt, img->N, ctx->in == PACT_BF16, ctx->out == PACT_BF16, ctx->ccfg, st);
+  CK(launch_merge(bt, img->N, ctx->in == PACT_BF16, ctx->out == PACT_BF16, ctx->ccfg, st));
   ctx->launches += 2;
   CK(cudaGetLastError());
   CK(cudaMemcpyAsync(img->counters, m.cnt, sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
@@ -510,7 +511,7 @@ pact_status pact_reduce(pact_ctx *ctx, const pact_image *imgs, int B, const pact
     CK(mark());
     launch_label(bt, cmaxN, bf, ROWS_ALL, st);      CK(mark());
     launch_lists(bt, cmaxN, st);                    CK(mark());
-    launch_merge(bt, cmaxN, bf, ctx->out == PACT_BF16, ctx->ccfg, st);  CK(mark());
+    CK(launch_merge(bt, cmaxN, bf, ctx->out == PACT_BF16, ctx->ccfg, st));  CK(mark());
     ctx->launches += 10;
     CK(cudaGetLastError());
     for (int b = 0; b < nb; ++b)

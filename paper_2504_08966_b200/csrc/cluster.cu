@@ -295,6 +295,7 @@ __global__ void __launch_bounds__(256) k_centers(const __grid_constant__ Batch b
     }
   }
   __syncwarp();
+  TL_POINT(bt.img[0], 10);
 
   // part 2: resolve
   int sweeps = 0, pending = 1;
@@ -356,8 +357,10 @@ __global__ void __launch_bounds__(256) k_centers(const __grid_constant__ Batch b
   }
 
   // part 3: every decision is final once all CTAs are here
+  TL_POINT(bt.img[0], 11);
   __threadfence();
   grid.sync();
+  TL_POINT(bt.img[0], 12);
   for (int item = gw; item < total; item += nwarps) {
     int b = 0;
     while (item >= qs[b + 1]) ++b;

@@ -61,7 +61,6 @@ struct ImgDesc {
   int32_t *blocklist;    // [ceil(N/256)][256] tokens of each block sorted by (cluster id, token)
   uint16_t *bstart;      // [ceil(N/256)][bstride] tokens of the block with a cluster id below c
   int32_t *csize;        // [Np] members of cluster c
-  int32_t *cbase;        // [Np] first scratch row of the clusters that are summed in several chunks
   int32_t *cticket;      // [Np] chunks of cluster c that are finished
   float *mpart;          // [N/8 + 2][d] chunk sums
   int32_t *cnt;          // [PACT_N_COUNTERS] + tickets: [16] global query, [19] member lists
@@ -105,8 +104,20 @@ struct TlScope {
   }
 };
 #define TL_SCOPE(im, kid) TlScope tl_scope_(im, kid)
+// a point inside a kernel: the time thread 0 of each CTA passes it, stored like a start time
+#define TL_POINT(im, kid)                                                                            \
+  do {                                                                                               \
+    const unsigned cta_ = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);            \
+    if ((im).tl && cta_ < kTlCtas && threadIdx.x == 0) {                                             \
+      unsigned long long t_;                                                                         \
+      asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_));                                          \
+      (im).tl[((size_t)(kid) * kTlCtas + cta_) * 2] = t_;                                            \
+      (im).tl[((size_t)(kid) * kTlCtas + cta_) * 2 + 1] = t_;                                        \
+    }                                                                                                \
+  } while (0)
 #else
 #define TL_SCOPE(im, kid)
+#define TL_POINT(im, kid)
 #endif
 
 // ---- element access ----------------------------------------------------------------------

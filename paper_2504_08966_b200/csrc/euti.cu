@@ -13,6 +13,7 @@
 // The kernels are short chains of dependent memory round trips; each issues all the loads it can
 // before it consumes the first.
 #include "kernels.cuh"
+#include "tma.cuh"
 
 namespace pact {
 
@@ -22,17 +23,22 @@ __device__ __forceinline__ double ld_cg_f64(const double *p) {
   return v;
 }
 
-constexpr int kPreThreads = 512;
-constexpr int kTokWarps = kPreThreads / 32;   // tokens per CTA of the token part of k_prepass
-constexpr int kQCtasMax = kQPartRows;         // CTAs that reduce Q
+constexpr int kPreConsumers = 8;                           // warps that reduce rows
+constexpr int kPreThreads = 32 * (1 + kPreConsumers);      // warp 0 issues the bulk copies
+constexpr int kPreStagesMax = 16;
+constexpr int kQCtasMax = kQPartRows;                      // CTAs that reduce Q
 
 // ---- Eq. 1 and the norms -----------------------------------------------------------------------
-// grid (GQ + ceil(maxN / 16), B), 512 threads.
+// grid (GQ + X, B), 288 threads.
 //  CTAs [0, GQ): column sums of a contiguous block of rows of Q; the last of them to finish adds
 //                the GQ partial sums in index order and writes the global query.
-//  other CTAs:   one warp per visual token: |h_i| (double) and 1 / |k_i| of the clustering key.
+//  other CTAs:   persistent, one per SM: CTA x takes a contiguous block of visual tokens.  Warp 0
+//                streams each token's hidden-state row and clustering-key row into a ring of shared
+//                memory slots with bulk copies (a steady depth of `stages` rows in flight per SM);
+//                warps 1-8 take the slots in turn: |h_i| (double) and 1 / |k_i|.
 template <typename T>
-__global__ void __launch_bounds__(kPreThreads) k_prepass(const __grid_constant__ Batch bt, int GQ) {
+__global__ void __launch_bounds__(kPreThreads) k_prepass(const __grid_constant__ Batch bt, int GQ, int stages,
+                                                          int slot_bytes) {
   using D = typename DistOf<T>::type;
   using rn_t = typename D::rn_t;
   constexpr int V = Vec<T>::N;
@@ -40,33 +46,76 @@ __global__ void __launch_bounds__(kPreThreads) k_prepass(const __grid_constant__
   TL_SCOPE(im, 0);
   const int t = threadIdx.x, lane = t & 31, w = t >> 5;
   if ((int)blockIdx.x >= GQ) {
-    const int tok = ((int)blockIdx.x - GQ) * kTokWarps + w;
-    if (tok >= im.N) return;
-    // every load of the token (key row, then hidden-state row) is issued before the first is used
-    constexpr int UK = 4;
-    const T *krow = im.Kc ? reinterpret_cast<const T *>(im.Kc) + (size_t)tok * im.ldKc : nullptr;
-    const int nvk = krow ? bt.d_k / V : 0;
-    uint4 kb[UK];
-#pragma unroll
-    for (int u = 0; u < UK; ++u)
-      if (lane + 32 * u < nvk) kb[u] = __ldg(reinterpret_cast<const uint4 *>(krow) + lane + 32 * u);
-    if (im.H) {
-      double nn = 1.0;
-      if (!(im.flags & PACT_FLAG_NO_NORM)) {
-        const T *hrow = reinterpret_cast<const T *>(im.H) + (size_t)(im.vis_start + tok) * im.ldH;
-        nn = sqrt(warp_sum(row_sumsq_lane<T, 16>(hrow, bt.d, lane)));
+    extern __shared__ __align__(128) unsigned char ring[];
+    __shared__ uint64_t full[kPreStagesMax], empty[kPreStagesMax];
+    __shared__ int abort_flag;
+    const int X = gridDim.x - GQ, x = blockIdx.x - GQ;
+    const int per = (im.N + X - 1) / X;
+    const int t0 = min(im.N, x * per), ntok = min(im.N, t0 + per) - t0;
+    const bool want_h = im.H && !(im.flags & PACT_FLAG_NO_NORM);
+    const bool want_k = im.Kc != nullptr;
+    const uint32_t hbytes = want_h ? (uint32_t)bt.d * sizeof(T) : 0u;
+    const uint32_t kbytes = want_k ? (uint32_t)bt.d_k * sizeof(T) : 0u;
+    if (ntok <= 0) return;
+    if (hbytes + kbytes == 0u) {                     // nothing to read: the norm factor is switched off
+      for (int i = t; i < ntok; i += kPreThreads) if (im.H) im.nrm[t0 + i] = 1.0;
+      return;
+    }
+    if (t == 0) {
+      for (int s = 0; s < stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+      abort_flag = 0;
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (w == 0) {
+      if (lane == 0) {
+        const T *H = reinterpret_cast<const T *>(im.H);
+        const T *Kc = reinterpret_cast<const T *>(im.Kc);
+        int i = 0;
+        bool ok = true;
+        const uint64_t keep = l2_policy_evict_last();   // the merge reads the hidden-state rows again
+        for (; i < ntok; ++i) {
+          const int s = i % stages;
+          if (!mbar_wait(&empty[s], ((i / stages) & 1) ^ 1)) { ok = false; break; }
+          unsigned char *dst = ring + (size_t)s * slot_bytes;
+          mbar_arrive_expect_tx(&full[s], hbytes + kbytes);
+          if (want_h) bulk_load_1d_hint(dst, H + (size_t)(im.vis_start + t0 + i) * im.ldH, hbytes, &full[s], keep);
+          if (want_k) bulk_load_1d(dst + hbytes, Kc + (size_t)(t0 + i) * im.ldKc, kbytes, &full[s]);
+        }
+        if (!ok) {
+          atomicExch(&abort_flag, 1);
+          // every copy that was issued lands before this CTA's shared memory is given up
+          const int armed = i < stages ? i : stages;
+          for (int k = 0; k < armed; ++k) {
+            const int j = i - 1 - k;
+            mbar_wait(&full[j % stages], (j / stages) & 1);
+          }
+        }
       }
-      if (lane == 0) im.nrm[tok] = nn;
+    } else {
+      const int cw = w - 1;
+      const int nvh = (int)(hbytes / 16), nvk = (int)(kbytes / 16);
+      for (int i = cw; i < ntok; i += kPreConsumers) {
+        const int s = i % stages;
+        if (!mbar_wait_warp(&full[s], (i / stages) & 1)) { atomicExch(&abort_flag, 1); break; }
+        const uint4 *src = reinterpret_cast<const uint4 *>(ring + (size_t)s * slot_bytes);
+        double acc_h = 0.0, acc_k = 0.0;
+        for (int v = lane; v < nvh; v += 32) sumsq_accumulate<T>(src[v], acc_h);
+        for (int v = lane; v < nvk; v += 32) sumsq_accumulate<T>(src[nvh + v], acc_k);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty[s]);       // the slot may be refilled
+        if (im.H) {
+          const double nn = want_h ? sqrt(warp_sum(acc_h)) : 1.0;
+          if (lane == 0) im.nrm[t0 + i] = nn;
+        }
+        if (want_k) {
+          const double ss = warp_sum(acc_k);
+          if (lane == 0) rn_tok<D>(im)[t0 + i] = (rn_t)(1.0 / sqrt(fmax(ss, 1e-40)));
+        }
+      }
     }
-    if (krow) {
-      double acc = 0.0;
-#pragma unroll
-      for (int u = 0; u < UK; ++u)
-        if (lane + 32 * u < nvk) sumsq_accumulate<T>(kb[u], acc);
-      if (nvk > 32 * UK) acc += row_sumsq_lane<T, 8>(krow, bt.d_k, lane, 32 * UK);
-      const double ss = warp_sum(acc);
-      if (lane == 0) rn_tok<D>(im)[tok] = (rn_t)(1.0 / sqrt(fmax(ss, 1e-40)));
-    }
+    __syncthreads();
+    if (t == 0 && abort_flag) atomicMin(&im.cnt[PACT_CNT_STATUS], (int)PACT_ERR_TIMEOUT);
     return;
   }
   if (!im.Q) return;
@@ -74,9 +123,10 @@ __global__ void __launch_bounds__(kPreThreads) k_prepass(const __grid_constant__
   const int chunk = (im.N + GQ - 1) / GQ;
   const int r0 = min(im.N, g * chunk), r1 = min(im.N, r0 + chunk);
   const int ncolv = bt.n_qcols / V;
-  const int cpp = min(ncolv, kPreThreads);   // column vectors per pass
-  const int groups = kPreThreads / cpp;      // row groups per pass
-  __shared__ double sm[kPreThreads * V];
+  constexpr int kQThreads = 256;                     // threads of a Q CTA that take part
+  const int cpp = min(ncolv, kQThreads);             // column vectors per pass
+  const int groups = kQThreads / cpp;                // row groups per pass
+  __shared__ double sm[kQThreads * V];
   const T *Q = reinterpret_cast<const T *>(im.Q);
   const int c = t % cpp, gi = t / cpp;
   constexpr int UQ = 8;
@@ -102,8 +152,10 @@ __global__ void __launch_bounds__(kPreThreads) k_prepass(const __grid_constant__
         }
       }
     }
+    if (t < kQThreads) {
 #pragma unroll
-    for (int k = 0; k < V; ++k) sm[t * V + k] = acc[k];
+      for (int k = 0; k < V; ++k) sm[t * V + k] = acc[k];
+    }
     __syncthreads();
     if (gi == 0 && cbase + c < ncolv) {
 #pragma unroll
@@ -170,37 +222,59 @@ __global__ void __launch_bounds__(kLogitThreads) k_logits(const __grid_constant_
   for (int c = t; c < bt.n_qcols; c += kLogitThreads) qg[(c % V) * nvq + c / V] = im.qg[c];
   __syncthreads();
   const int vph = d_h / V;                                  // vectors per head
+  for (int j = 0; j < n_qh; ++j) {
+    // the tokens of this warp give independent chains of multiply-adds; their sums are reduced together
+    double acc[kLogitTpw][UK];
 #pragma unroll
-  for (int i = 0; i < kLogitTpw; ++i) {
-    const int lr = w * kLogitTpw + i;                       // token within the CTA
-    if (r0 + lr >= r1) break;
-    const uint4 *krow = reinterpret_cast<const uint4 *>(K + (size_t)(r0 + lr) * im.ldKe);
-    for (int j = 0; j < n_qh; ++j) {
-      double acc = 0.0;
-      if (use_query) {
-        const int kv = (j * bt.n_kvh) / n_qh;
-        const int vshift = (j - kv) * vph;                  // key-row vector v pairs with query vector v + vshift
+    for (int i = 0; i < kLogitTpw; ++i)
 #pragma unroll
-        for (int u = 0; u < UK; ++u) {
-          const int v = lane + 32 * u;
-          if (v < nv && v / vph == kv) {
+      for (int u = 0; u < UK; ++u) acc[i][u] = 0.0;
+    if (use_query) {
+      const int kv = (j * bt.n_kvh) / n_qh;
+      const int vshift = (j - kv) * vph;                    // key-row vector v pairs with query vector v + vshift
+#pragma unroll
+      for (int u = 0; u < UK; ++u) {
+        const int v = lane + 32 * u;
+        if (v < nv && v / vph == kv) {
+          double qv[V];
+#pragma unroll
+          for (int k = 0; k < V; ++k) qv[k] = qg[k * nvq + v + vshift];
+#pragma unroll
+          for (int i = 0; i < kLogitTpw; ++i) {
             float x[V];
             widen_vec<T>(kb[i][u], x);
 #pragma unroll
-            for (int k = 0; k < V; ++k) acc = fma((double)x[k], qg[k * nvq + v + vshift], acc);
+            for (int k = 0; k < V; ++k) acc[i][u] = fma((double)x[k], qv[k], acc[i][u]);
           }
         }
-        for (int v = lane + 32 * UK; v < nv; v += 32) {     // rows wider than the preloaded part
-          if (v / vph == kv) {
-            float x[V];
-            widen_vec<T>(__ldg(krow + v), x);
-#pragma unroll
-            for (int k = 0; k < V; ++k) acc = fma((double)x[k], qg[k * nvq + v + vshift], acc);
-          }
-        }
-        acc = warp_sum(acc);
       }
-      if (lane == 0) lg[lr * n_qh + j] = acc;
+      for (int v = lane + 32 * UK; v < nv; v += 32) {       // rows wider than the preloaded part
+        if (v / vph == kv) {
+#pragma unroll
+          for (int i = 0; i < kLogitTpw; ++i) {
+            const int rr = min(r0 + w * kLogitTpw + i, im.N - 1);
+            float x[V];
+            widen_vec<T>(__ldg(reinterpret_cast<const uint4 *>(K + (size_t)rr * im.ldKe) + v), x);
+#pragma unroll
+            for (int k = 0; k < V; ++k) acc[i][0] = fma((double)x[k], qg[k * nvq + v + vshift], acc[i][0]);
+          }
+        }
+      }
+    }
+    double tot[kLogitTpw];
+#pragma unroll
+    for (int i = 0; i < kLogitTpw; ++i) {
+      tot[i] = acc[i][0];
+#pragma unroll
+      for (int u = 1; u < UK; ++u) tot[i] += acc[i][u];
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+      for (int i = 0; i < kLogitTpw; ++i) tot[i] += __shfl_xor_sync(0xffffffffu, tot[i], o);
+    if (lane == 0) {
+#pragma unroll
+      for (int i = 0; i < kLogitTpw; ++i) lg[(w * kLogitTpw + i) * n_qh + j] = tot[i];
     }
   }
   __syncthreads();
@@ -284,11 +358,13 @@ __device__ __forceinline__ uint32_t score_key(float s) {
   return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
-// grid (X, B), 1024 threads; dynamic smem: (keys_in_smem) N keys, then own_cap token indices.
+// grid (X, B), 1024 threads; dynamic smem: own_cap token indices, then (KPT == 0 and keys_in_smem) N keys.
 // Every CTA computes the same threshold and the same list positions; CTA b writes the list entries of
 // its block of tokens, and (do_gather) copies its block of survivor rows into Kp and their inverse
 // norms into rnk, and clears its share of the arrays that later kernels accumulate into.
-template <typename T>
+// KPT > 0: thread t keeps the keys of tokens [t KPT, t KPT + KPT) in registers (N <= 1024 KPT);
+// KPT == 0: any N, keys in shared memory when they fit, else re-read from the scores.
+template <typename T, int KPT>
 __global__ void __launch_bounds__(1024) k_select_gather(const __grid_constant__ Batch bt, int do_gather,
                                                         int keys_in_smem, int own_cap) {
   using D = typename DistOf<T>::type;
@@ -297,16 +373,29 @@ __global__ void __launch_bounds__(1024) k_select_gather(const __grid_constant__ 
   const int t = threadIdx.x, lane = t & 31, w = t >> 5;
   const int N = im.N;
   extern __shared__ uint32_t dsm[];
-  uint32_t *skey = dsm;                                     // [N] when keys_in_smem
-  int *own = reinterpret_cast<int *>(dsm + (keys_in_smem ? N : 0));   // [own_cap]
+  int *own = reinterpret_cast<int *>(dsm);                  // [own_cap]
+  uint32_t *skey = dsm + own_cap;                           // [N] when KPT == 0 and keys_in_smem
   __shared__ int hist[256];
   __shared__ int warp_tot[32];
   __shared__ uint32_t wmin[32], wmax[32];
   __shared__ uint32_t s_prefix;
   __shared__ int s_k;
+  constexpr int KR = KPT > 0 ? KPT : 1;
+  const int CH = KPT > 0 ? KPT : (N + 1023) / 1024;         // tokens per thread, contiguous
+  const int i0 = min(N, t * CH), i1 = min(N, i0 + CH);
+  const int cnt_mine = i1 - i0;
 
-  if (keys_in_smem)
+  // keys of this thread's tokens
+  uint32_t kreg[KR];
+  if (KPT > 0) {
+    float sc[KR];
+#pragma unroll
+    for (int j = 0; j < KR; ++j) sc[j] = j < cnt_mine ? __ldg(im.score + i0 + j) : 0.f;
+#pragma unroll
+    for (int j = 0; j < KR; ++j) kreg[j] = score_key(sc[j]);
+  } else if (keys_in_smem) {
     for (int i = t; i < N; i += 1024) skey[i] = score_key(im.score[i]);
+  }
   if (do_gather) {   // per-call initialisation, spread over the grid
     const int gt = blockIdx.x * 1024 + t, gs = gridDim.x * 1024;
     for (int r = gt; r < im.Np; r += gs) { im.rho_fix[r] = 0ull; im.csize[r] = 0; im.cticket[r] = 0; }
@@ -316,14 +405,21 @@ __global__ void __launch_bounds__(1024) k_select_gather(const __grid_constant__ 
   if (t == 0) s_k = im.m_target;
   if (t < 256) hist[t] = 0;
   __syncthreads();
-  auto key = [&](int i) -> uint32_t { return keys_in_smem ? skey[i] : score_key(im.score[i]); };
+  // j-th key of this thread (j < cnt_mine)
+  auto key = [&](int j) -> uint32_t {
+    if (KPT > 0) return kreg[j < KR ? j : 0];
+    return keys_in_smem ? skey[i0 + j] : score_key(im.score[i0 + j]);
+  };
 
-  // The bits above the highest bit in which two keys differ are common to all keys and need no pass.
-  const int rounds = (N + 1023) / 1024;
+  // Keys are taken relative to the smallest one: that spreads them evenly over the digits of the first
+  // pass (raw float bits of scores that span a few binades share most of their top bits), and the bits
+  // above the highest one in which two keys differ need no pass.
   uint32_t kmin = 0xffffffffu, kmax = 0u;
-  for (int it = 0; it < rounds; ++it) {
-    const int i = it * 1024 + t;
-    if (i < N) { const uint32_t kk = key(i); kmin = min(kmin, kk); kmax = max(kmax, kk); }
+  if (KPT > 0) {
+#pragma unroll
+    for (int j = 0; j < KR; ++j) if (j < cnt_mine) { kmin = min(kmin, kreg[j]); kmax = max(kmax, kreg[j]); }
+  } else {
+    for (int j = 0; j < cnt_mine; ++j) { const uint32_t kk = key(j); kmin = min(kmin, kk); kmax = max(kmax, kk); }
   }
   kmin = __reduce_min_sync(0xffffffffu, kmin);
   kmax = __reduce_max_sync(0xffffffffu, kmax);
@@ -331,8 +427,9 @@ __global__ void __launch_bounds__(1024) k_select_gather(const __grid_constant__ 
   __syncthreads();
   kmin = __reduce_min_sync(0xffffffffu, wmin[lane]);
   kmax = __reduce_max_sync(0xffffffffu, wmax[lane]);
-  const int top = 32 - __clz(kmin ^ kmax);                  // low bits that vary (0: all keys are equal)
-  if (t == 0) s_prefix = top >= 32 ? 0u : (kmin >> top) << top;
+  const uint32_t kbase = kmin;
+  const int top = 32 - __clz(kmax - kbase);                 // bits of the largest relative key (0: all keys equal)
+  if (t == 0) s_prefix = 0u;
   __syncthreads();
 
   // radix select of the (m_target + 1)-th smallest key over the varying bits, up to 8 bits per pass
@@ -341,10 +438,15 @@ __global__ void __launch_bounds__(1024) k_select_gather(const __grid_constant__ 
     const uint32_t dmask = (1u << (hi - lo)) - 1u;
     const uint32_t above = hi >= 32 ? 0u : ~((1u << hi) - 1u);   // bits already fixed
     const uint32_t prefix = s_prefix;
-    for (int it = 0; it < rounds; ++it) {
-      const int i = it * 1024 + t;
-      if (i < N) {
-        const uint32_t kk = key(i);
+    if (KPT > 0) {
+#pragma unroll
+      for (int j = 0; j < KR; ++j) {
+        const uint32_t kk = kreg[j] - kbase;
+        if (j < cnt_mine && (kk & above) == (prefix & above)) atomicAdd(&hist[(kk >> lo) & dmask], 1);
+      }
+    } else {
+      for (int j = 0; j < cnt_mine; ++j) {
+        const uint32_t kk = key(j) - kbase;
         if ((kk & above) == (prefix & above)) atomicAdd(&hist[(kk >> lo) & dmask], 1);
       }
     }
@@ -380,13 +482,20 @@ __global__ void __launch_bounds__(1024) k_select_gather(const __grid_constant__ 
     }
     __syncthreads();
   }
-  const uint32_t tau_key = s_prefix;
+  const uint32_t tau_key = s_prefix + kbase;
 
-  // ordered compaction: thread t owns tokens [t * CH, t * CH + CH)
-  const int CH = (N + 1023) / 1024;
-  const int i0 = min(N, t * CH), i1 = min(N, i0 + CH);
+  // ordered compaction over the contiguous blocks of tokens
+  uint32_t keptbits = 0u;
+  if (KPT > 0) {
+#pragma unroll
+    for (int j = 0; j < KR; ++j) if (j < cnt_mine && kreg[j] >= tau_key) keptbits |= 1u << j;
+  } else {
+    // more than 32 tokens per thread only beyond 32768 tokens: the bits are recomputed below then
+    for (int j = 0; j < cnt_mine && j < 32; ++j) if (key(j) >= tau_key) keptbits |= 1u << j;
+  }
   int mine = 0;
-  for (int i = i0; i < i1; ++i) mine += key(i) >= tau_key;
+  if (KPT > 0 || CH <= 32) mine = __popc(keptbits);
+  else for (int j = 0; j < cnt_mine; ++j) mine += key(j) >= tau_key;
   int incl = mine;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -413,17 +522,21 @@ __global__ void __launch_bounds__(1024) k_select_gather(const __grid_constant__ 
   const int w0 = blockIdx.x * tpc, w1 = min(N, w0 + tpc);
   const int rpc = (q + gridDim.x - 1) / gridDim.x;          // survivor rows this CTA gathers
   const int g0 = min(q, (int)blockIdx.x * rpc), g1 = min(q, g0 + rpc);
-  for (int i = i0; i < i1; ++i) {
-    const bool kp = key(i) >= tau_key;
-    if (i >= w0 && i < w1) {
-      im.keep[i] = kp ? 1 : 0;
-      if (im.keep_user) im.keep_user[i] = kp ? 1 : 0;
-      if (kp) { im.kept_idx[before] = i; im.slot[i] = before; }
-      else { im.pruned_idx[i - before] = i; im.slot[i] = -1 - (i - before); }
-    }
-    if (kp) {
-      if (do_gather && before >= g0 && before < g1 && before - g0 < own_cap) own[before - g0] = i;
-      ++before;
+  const bool touches = (i0 < w1 && i1 > w0) || (do_gather && before < g1 && before + mine > g0);
+  if (touches) {
+    for (int j = 0; j < cnt_mine; ++j) {
+      const int i = i0 + j;
+      const bool kp = (KPT > 0 || CH <= 32) ? ((keptbits >> j) & 1u) != 0u : key(j) >= tau_key;
+      if (i >= w0 && i < w1) {
+        im.keep[i] = kp ? 1 : 0;
+        if (im.keep_user) im.keep_user[i] = kp ? 1 : 0;
+        if (kp) { im.kept_idx[before] = i; im.slot[i] = before; }
+        else { im.pruned_idx[i - before] = i; im.slot[i] = -1 - (i - before); }
+      }
+      if (kp) {
+        if (do_gather && before >= g0 && before < g1 && before - g0 < own_cap) own[before - g0] = i;
+        ++before;
+      }
     }
   }
   if (blockIdx.x == 0 && t == 0) {
@@ -458,19 +571,31 @@ __global__ void __launch_bounds__(1024) k_select_gather(const __grid_constant__ 
 namespace {
 int g_sm_count = 148;
 size_t g_smem_optin = 48 * 1024;
+size_t g_prepass_ring = 40 * 1024;           // bytes of shared memory the prepass may use for its ring
 constexpr size_t kSelectReserve = 4096;      // static shared memory of k_select_gather, rounded up
 
 int q_ctas(int maxN) {
-  const int g = (maxN + 127) / 128;
+  const int g = (maxN + 63) / 64;
   return g < 1 ? 1 : (g > kQCtasMax ? kQCtasMax : g);
 }
 }  // namespace
 
 void launch_prepass(const Batch &bt, int maxN, bool bf16, cudaStream_t st) {
   const int GQ = q_ctas(maxN);
-  dim3 grid(GQ + (maxN + kTokWarps - 1) / kTokWarps, bt.B);
-  if (bf16) k_prepass<__nv_bfloat16><<<grid, kPreThreads, 0, st>>>(bt, GQ);
-  else k_prepass<float><<<grid, kPreThreads, 0, st>>>(bt, GQ);
+  const int elt = bf16 ? 2 : 4;
+  int slot = (bt.d + bt.d_k) * elt;
+  slot = (slot + 127) / 128 * 128;
+  int stages = (int)(g_prepass_ring / (size_t)slot);
+  if (stages > kPreStagesMax) stages = kPreStagesMax;
+  if (stages < 2) stages = 2;                      // pact_create has checked that two slots fit
+  int X = g_sm_count / bt.B;
+  if (X < 1) X = 1;
+  const int cap = (maxN + 7) / 8;                  // at least 8 tokens per CTA
+  if (X > cap) X = cap;
+  dim3 grid(GQ + X, bt.B);
+  const size_t smem = (size_t)stages * slot;
+  if (bf16) k_prepass<__nv_bfloat16><<<grid, kPreThreads, smem, st>>>(bt, GQ, stages, slot);
+  else k_prepass<float><<<grid, kPreThreads, smem, st>>>(bt, GQ, stages, slot);
 }
 
 void launch_logits(const Batch &bt, int maxN, bool bf16, cudaStream_t st) {
@@ -484,7 +609,8 @@ void launch_scores(const Batch &bt, int maxN, cudaStream_t st) {
   k_scores<<<dim3((maxN + 255) / 256, bt.B), 256, 0, st>>>(bt);
 }
 
-void launch_select_gather(const Batch &bt, int maxN, bool bf16, bool gather, cudaStream_t st) {
+template <typename T>
+static void launch_select_t(const Batch &bt, int maxN, bool gather, cudaStream_t st) {
   int X = 1;
   if (gather) {
     X = g_sm_count / bt.B;
@@ -494,11 +620,20 @@ void launch_select_gather(const Batch &bt, int maxN, bool bf16, bool gather, cud
   }
   const int own_cap = gather ? (maxN + X - 1) / X + 1 : 0;
   size_t sm = (size_t)own_cap * sizeof(int);
-  const bool in_smem = sm + (size_t)maxN * 4 + kSelectReserve <= g_smem_optin;
-  if (in_smem) sm += (size_t)maxN * 4;
   dim3 grid(X, bt.B);
-  if (bf16) k_select_gather<__nv_bfloat16><<<grid, 1024, sm, st>>>(bt, gather ? 1 : 0, in_smem ? 1 : 0, own_cap);
-  else k_select_gather<float><<<grid, 1024, sm, st>>>(bt, gather ? 1 : 0, in_smem ? 1 : 0, own_cap);
+  const int g = gather ? 1 : 0;
+  if (maxN <= 8 * 1024) k_select_gather<T, 8><<<grid, 1024, sm, st>>>(bt, g, 0, own_cap);
+  else if (maxN <= 16 * 1024) k_select_gather<T, 16><<<grid, 1024, sm, st>>>(bt, g, 0, own_cap);
+  else {
+    const bool in_smem = sm + (size_t)maxN * 4 + kSelectReserve <= g_smem_optin;
+    if (in_smem) sm += (size_t)maxN * 4;
+    k_select_gather<T, 0><<<grid, 1024, sm, st>>>(bt, g, in_smem ? 1 : 0, own_cap);
+  }
+}
+
+void launch_select_gather(const Batch &bt, int maxN, bool bf16, bool gather, cudaStream_t st) {
+  if (bf16) launch_select_t<__nv_bfloat16>(bt, maxN, gather, st);
+  else launch_select_t<float>(bt, maxN, gather, st);
 }
 
 cudaError_t select_configure() {
@@ -512,13 +647,22 @@ cudaError_t select_configure() {
   if (e != cudaSuccess) return e;
   g_smem_optin = (size_t)v;
   const int dyn = (int)(g_smem_optin - kSelectReserve);
-  e = cudaFuncSetAttribute(k_select_gather<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn);
+  e = cudaFuncSetAttribute(k_select_gather<__nv_bfloat16, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(k_select_gather<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn);
+  return cudaFuncSetAttribute(k_select_gather<float, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn);
 }
 
-cudaError_t euti_configure(int n_qcols, int n_qh) {
+cudaError_t euti_configure(int n_qcols, int n_qh, int d, int d_k, int elt) {
   cudaError_t e = select_configure();
+  if (e != cudaSuccess) return e;
+  // every CTA of the launch reserves the ring; two of them (a streaming one and a Q-reducing one) must
+  // fit on an SM together
+  g_prepass_ring = g_smem_optin > 200 * 1024 ? 92 * 1024 : g_smem_optin / 3;
+  const size_t slot = ((size_t)(d + d_k) * elt + 127) / 128 * 128;
+  if (2 * slot > g_prepass_ring) return cudaErrorInvalidConfiguration;
+  e = cudaFuncSetAttribute(k_prepass<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g_prepass_ring);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(k_prepass<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g_prepass_ring);
   if (e != cudaSuccess) return e;
   const size_t sm = (size_t)(n_qcols + kRowsPerCta * n_qh) * sizeof(double);
   if (sm > g_smem_optin) return cudaErrorInvalidConfiguration;

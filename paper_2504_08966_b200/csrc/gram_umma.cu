@@ -14,6 +14,7 @@
 #include <cuda.h>
 
 #include "kernels.cuh"
+#include "tma.cuh"
 
 namespace pact {
 
@@ -27,51 +28,11 @@ constexpr int A_BYTES = BM * BK * 2;
 constexpr int B_BYTES = BN * BK * 2;
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int TMEM_COLS = 2 * BN; // 512: all of an SM's tensor memory
-constexpr unsigned long long kWaitNs = 1000000000ull;   // one second per wait, then give up
 
 struct TmapSet {
   CUtensorMap a[kMaxBatchPerLaunch];
   CUtensorMap b[kMaxBatchPerLaunch];
 };
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ unsigned long long global_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-// Bounded wait: false when kWaitNs of wall time have passed without the phase completing.
-__device__ __noinline__ bool mbar_wait_slow(uint64_t *bar, uint32_t parity) {
-  const unsigned long long t0 = global_ns();
-  for (uint32_t i = 0;; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 255u) == 255u && global_ns() - t0 > kWaitNs) return false;
-  }
-}
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
-  for (int i = 0; i < 64; ++i)
-    if (mbar_try_wait(bar, parity)) return true;
-  return mbar_wait_slow(bar, parity);
-}
 
 __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, uint64_t *bar, int x, int y) {
   asm volatile(
@@ -303,7 +264,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
       __syncwarp();
       reinterpret_cast<float4 *>(rn_col)[lane] = r4;
       __syncwarp();
-      if (!__all_sync(0xffffffffu, mbar_wait(&sh.acc_full[a], (tcount >> 1) & 1))) { ok = false; break; }
+      if (!mbar_wait_warp(&sh.acc_full[a], (tcount >> 1) & 1)) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + a * BN + half * HALF + ((uint32_t)(qd * 32) << 16);
       unsigned long long rowsum = 0ull;

@@ -10,13 +10,13 @@ constexpr int kMergeMaxD = 256 * 4 * 8;   // widest hidden state the merge kerne
 enum RowMode { ROWS_ALL = 0, ROWS_KEPT_LIST = 1, ROWS_PRUNED_LIST = 2 };
 
 // euti.cu
-constexpr int kQPartRows = 32;            // most partial sums of Q the prepass writes per image
+constexpr int kQPartRows = 64;            // most partial sums of Q the prepass writes per image
 void launch_prepass(const Batch &bt, int maxN, bool bf16, cudaStream_t st);
 void launch_logits(const Batch &bt, int maxN, bool bf16, cudaStream_t st);
 void launch_scores(const Batch &bt, int maxN, cudaStream_t st);
 // threshold + ordered compaction; gather: also copy the survivor keys and clear the accumulators
 void launch_select_gather(const Batch &bt, int maxN, bool bf16, bool gather, cudaStream_t st);
-cudaError_t euti_configure(int n_qcols, int n_qh);
+cudaError_t euti_configure(int n_qcols, int n_qh, int d, int d_k, int elt);
 cudaError_t select_configure();            // what launch_select_gather needs, once per device
 
 // cluster.cu
@@ -44,6 +44,8 @@ cudaError_t launch_assign_umma(const Batch &bt, int maxN, bool kept_rows, const 
 // merge.cu
 // member lists from label[]; csize and cticket must be zero
 void launch_lists(const Batch &bt, int maxN, cudaStream_t st);
-void launch_merge(const Batch &bt, int maxN, bool in_bf16, bool out_bf16, const ClusterCfg &cfg, cudaStream_t st);
+cudaError_t launch_merge(const Batch &bt, int maxN, bool in_bf16, bool out_bf16, const ClusterCfg &cfg, cudaStream_t st);
+cudaError_t merge_configure();
+int merge_max_tokens(int d, int elt);      // largest N the merge kernel takes (its chunk offsets live in shared memory)
 
 }  // namespace pact
