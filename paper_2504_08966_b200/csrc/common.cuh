@@ -105,10 +105,11 @@ struct TlScope {
 };
 #define TL_SCOPE(im, kid) TlScope tl_scope_(im, kid)
 // a point inside a kernel: the time thread 0 of each CTA passes it, stored like a start time
-#define TL_POINT(im, kid)                                                                            \
+#define TL_POINT(im, kid) TL_POINT_IF(im, kid, threadIdx.x == 0)
+#define TL_POINT_IF(im, kid, cond)                                                                   \
   do {                                                                                               \
     const unsigned cta_ = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);            \
-    if ((im).tl && cta_ < kTlCtas && threadIdx.x == 0) {                                             \
+    if ((im).tl && cta_ < kTlCtas && (cond)) {                                             \
       unsigned long long t_;                                                                         \
       asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_));                                          \
       (im).tl[((size_t)(kid) * kTlCtas + cta_) * 2] = t_;                                            \
@@ -118,6 +119,7 @@ struct TlScope {
 #else
 #define TL_SCOPE(im, kid)
 #define TL_POINT(im, kid)
+#define TL_POINT_IF(im, kid, cond)
 #endif
 
 // ---- element access ----------------------------------------------------------------------

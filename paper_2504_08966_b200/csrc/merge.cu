@@ -61,7 +61,6 @@ template <> struct Raw8<float> {
   }
 };
 
-constexpr int kMergeThreads = 256;
 constexpr int kListBlock = 256;      // tokens per block of the member lists
 constexpr int kChunk = 16;           // members summed by one work item
 
@@ -123,51 +122,35 @@ __global__ void __launch_bounds__(kListBlock) k_lists(const __grid_constant__ Ba
 }
 
 // ---- Eq. 10 ------------------------------------------------------------------------------------------
-// Persistent grid (X, B), one CTA per SM, 288 threads.  Work units are the chunks (kChunk members of one
-// cluster, ascending token order) followed by the text rows; CTA x takes units x, x + X, ...
-//  warp 0     looks up the members of each unit and streams their hidden-state rows, whole rows, into a
-//             ring of shared-memory slots with bulk copies: a steady depth of `stages` rows in flight
-//             whatever the cluster sizes are;
-//  warps 1-8  own a slice of the columns each; they take the slots in order, add their slice in float
-//             and at the end of a unit divide and store it.
-// A cluster of one chunk is finished on the spot; otherwise the chunk sums go to scratch and the CTA that
-// finishes the cluster's last chunk adds them in chunk order.  Every wait is bounded.
-constexpr int kMrgConsumers = 8;
-constexpr int kMrgThreads = 32 * (1 + kMrgConsumers);
-constexpr int kMrgStagesMax = 32;
-constexpr int kTabUnits = 32;                      // units a CTA looks up before it streams them
-constexpr int kMrgVpl = kMergeMaxD / 8 / (32 * kMrgConsumers);   // 8-column groups per consumer lane
+// Grid (X, B) with three CTAs of 256 threads per SM.  Work units are the chunks (kChunk members of one
+// cluster, ascending token order) followed by the text rows; CTA x takes units x, x + X, ...  For a unit
+// the CTA looks up the members (thread = block of the member lists), then every thread adds its columns
+// of the member rows in float with kMrgRows rows in flight, divides and stores.  A cluster of one chunk
+// is finished on the spot; otherwise the chunk sums go to scratch and the CTA that finishes the cluster's
+// last chunk adds them in chunk order.  Plain 16-byte loads: many small CTAs keep enough of them in
+// flight, and a CTA that waits on its look-up loads does not hold back the others.
+constexpr int kMrgThreads = 256;
+constexpr int kMrgRows = 4;                        // member rows in flight per thread
+constexpr int kMrgVpl = kMergeMaxD / 8 / kMrgThreads;   // 8-column groups per thread at the widest d
 
-__device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kMrgConsumers * 32) : "memory"); }
-
-template <typename T, typename O>
-__global__ void __launch_bounds__(kMrgThreads, 1) k_merge(const __grid_constant__ Batch bt, int stages, int slot_bytes,
-                                                         int ring_off) {
+template <typename T, typename O, int VPL>
+__global__ void __launch_bounds__(kMrgThreads, (VPL <= 2 && sizeof(T) == 2) ? 3 : 1)
+k_merge(const __grid_constant__ Batch bt) {
   const ImgDesc &im = bt.img[blockIdx.y];
   TL_SCOPE(im, 9);
   const int t = threadIdx.x, lane = t & 31, w = t >> 5;
-  extern __shared__ __align__(128) unsigned char dsm[];
-  int *chunk_off = reinterpret_cast<int *>(dsm);   // [C + 1] first chunk of cluster c
-  unsigned char *ring = dsm + ring_off;
-  __shared__ uint64_t full[kMrgStagesMax], empty[kMrgStagesMax];
+  extern __shared__ int chunk_off[];               // [C + 1] first chunk of cluster c
   __shared__ int wsum[kMrgThreads / 32];
-  __shared__ int s_carry, s_last, abort_flag;
-  __shared__ int mtab[kTabUnits][kChunk];          // members of the units of this round
-  __shared__ int meta[kTabUnits][8];               // cluster, chunk, chunks of the cluster, size, members, output row, centre row
+  __shared__ int s_carry, s_last;
+  __shared__ int members[kChunk];
   const int C = *im.C_ptr;
   const int n_text = im.n_total - im.N;
   const int d = bt.d, ng = d / 8;
   const bool center_only = (im.flags & PACT_FLAG_CENTER_ONLY) != 0;
   const T *H = reinterpret_cast<const T *>(im.H);
   O *Ho = reinterpret_cast<O *>(im.H_out);
-  const uint32_t row_bytes = (uint32_t)d * sizeof(T);
   if (blockIdx.x == 0 && t == 0) im.cnt[PACT_CNT_N_OUT] = n_text + C;
-  if (t == 0) {
-    for (int s = 0; s < stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kMrgConsumers); }
-    abort_flag = 0;
-    s_carry = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
+  if (t == 0) s_carry = 0;
   __syncthreads();
   // chunk offsets: exclusive prefix sum of the chunks per cluster
   for (int base = 0; base < C; base += kMrgThreads) {
@@ -196,186 +179,154 @@ __global__ void __launch_bounds__(kMrgThreads, 1) k_merge(const __grid_constant_
   const int n_units = n_chunks + n_text;
   const int nblk = (im.N + kListBlock - 1) / kListBlock;
 
-  // The units of this CTA are handled in rounds of up to kTabUnits.  In a round all warps first look up
-  // the units' clusters and members (short chains of dependent loads, issued by every CTA at the same
-  // time while no rows are in flight); then warp 0 streams the rows and warps 1-8 reduce them.
-  const int my_units = n_units > (int)blockIdx.x ? (n_units - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
-  int it_p = 0, it_c = 0;                          // rows issued / consumed so far
-  bool ok = true;
-  for (int round0 = 0; round0 < my_units; round0 += kTabUnits) {
-    const int nu = min(kTabUnits, my_units - round0);
-    for (int ui = w; ui < nu; ui += kMrgThreads / 32) {
-      const int u = blockIdx.x + (round0 + ui) * gridDim.x;
-      int c = -1, k = 0, nch = 1, size = 1, nm = 1, dst, ptok;
-      if (u >= n_chunks) {                         // a text row
-        const int tr = u - n_chunks;
-        const int src = tr < im.vis_start ? tr : tr + im.N;
-        dst = tr < im.vis_start ? tr : tr + C;
-        ptok = src;
-        if (lane == 0) mtab[ui][0] = src - im.vis_start;   // relative to the visual span
-      } else {
-        int lo = 0, hi = C - 1;                    // last c with chunk_off[c] <= u
-        while (lo < hi) {
-          const int mid = (lo + hi + 1) >> 1;
-          if (chunk_off[mid] <= u) lo = mid; else hi = mid - 1;
-        }
-        c = lo;
-        k = u - chunk_off[c];
-        nch = chunk_off[c + 1] - chunk_off[c];
-        size = im.csize[c];
-        const int ctok = im.cidx_ptr[c];
-        dst = im.vis_start + c;
-        ptok = im.vis_start + ctok;
-        if (center_only) {
-          if (lane == 0) mtab[ui][0] = ctok;
-        } else {
-          const int m0 = k * kChunk, m1 = min(size, m0 + kChunk);
-          nm = m1 - m0;
-          int carry = 0;
-          for (int bb0 = 0; bb0 < nblk && carry < m1; bb0 += 32) {   // lane = block of the member lists
-            const int bb = bb0 + lane;
-            int s0 = 0, cntb = 0;
-            if (bb < nblk) {
-              const uint16_t *row = im.bstart + (size_t)bb * im.bstride;
-              s0 = row[c];
-              cntb = (int)row[c + 1] - s0;
-            }
-            int x = cntb;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-              const int y = __shfl_up_sync(0xffffffffu, x, o);
-              if (lane >= o) x += y;
-            }
-            const int off = carry + x - cntb;      // list position of this block's first member
-            const int a0 = max(off, m0), a1 = min(off + cntb, m1);
-            for (int m = a0; m < a1; ++m) mtab[ui][m - m0] = im.blocklist[(size_t)bb * kListBlock + s0 + (m - off)];
-            carry += __shfl_sync(0xffffffffu, x, 31);
-          }
-        }
+  // units are handed out first come, first served (the order does not change any result)
+  __shared__ int s_next;
+  int u = blockIdx.x;
+  while (u < n_units) {
+    int c = -1, k = 0, nch = 1, size = 1, nm = 1, dst, ptok;
+    __syncthreads();                               // members, wsum and s_next of the previous unit are consumed
+    if (t == 0) s_next = gridDim.x + atomicAdd(&im.cnt[21], 1);   // needed only after this unit's rows
+    if (u >= n_chunks) {                           // a text row
+      const int tr = u - n_chunks;
+      const int src = tr < im.vis_start ? tr : tr + im.N;
+      dst = tr < im.vis_start ? tr : tr + C;
+      ptok = src;
+      if (t == 0) members[0] = src - im.vis_start; // relative to the visual span
+    } else {
+      int lo = 0, hi = C - 1;                      // last c with chunk_off[c] <= u
+      while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (chunk_off[mid] <= u) lo = mid; else hi = mid - 1;
       }
-      if (lane == 0) {
-        int *mt = meta[ui];
-        mt[0] = c; mt[1] = k; mt[2] = nch; mt[3] = size; mt[4] = nm; mt[5] = dst; mt[6] = ptok;
+      c = lo;
+      k = u - chunk_off[c];
+      nch = chunk_off[c + 1] - chunk_off[c];
+      size = im.csize[c];
+      const int ctok = im.cidx_ptr[c];
+      dst = im.vis_start + c;
+      ptok = im.vis_start + ctok;
+      if (center_only) {
+        if (t == 0) members[0] = ctok;
+      } else {
+        const int m0 = k * kChunk, m1 = min(size, m0 + kChunk);
+        nm = m1 - m0;
+        int carry = 0;
+        for (int bb0 = 0; bb0 < nblk; bb0 += kMrgThreads) {   // thread = block of the member lists
+          const int bb = bb0 + t;
+          int s0 = 0, cntb = 0;
+          if (bb < nblk) {                         // does not wait for the cluster size
+            const uint16_t *row = im.bstart + (size_t)bb * im.bstride;
+            s0 = row[c];
+            cntb = (int)row[c + 1] - s0;
+          }
+          int x = cntb;
+#pragma unroll
+          for (int o = 1; o < 32; o <<= 1) {
+            const int y = __shfl_up_sync(0xffffffffu, x, o);
+            if (lane >= o) x += y;
+          }
+          if (bb0 > 0) __syncthreads();            // wsum of the previous round is consumed
+          if (lane == 31) wsum[w] = x;
+          __syncthreads();
+          int off = carry, tot = 0;
+#pragma unroll
+          for (int q = 0; q < kMrgThreads / 32; ++q) { if (q < w) off += wsum[q]; tot += wsum[q]; }
+          off += x - cntb;                         // list position of this block's first member
+          const int a0 = max(off, m0), a1 = min(off + cntb, m1);
+          for (int m = a0; m < a1; ++m) members[m - m0] = im.blocklist[(size_t)bb * kListBlock + s0 + (m - off)];
+          carry += tot;
+          if (carry >= m1) break;                  // uniform
+        }
       }
     }
     __syncthreads();
-    if (w == 0) {
-      // ---------------- producer ----------------
-      // the lanes issue the rows of a unit side by side (copies issued by one thread complete one after
-      // the other); slot order is the row order, which the consumers follow
-      if (ok) {
-        const uint64_t once = l2_policy_evict_first();  // last use of these rows
-        for (int ui = 0; ok && ui < nu; ++ui) {
-          const int nm = meta[ui][4];
-          bool lane_ok = true;
-          if (lane < nm) {
-            const int itl = it_p + lane, s = itl % stages;
-            lane_ok = mbar_wait(&empty[s], ((itl / stages) & 1) ^ 1);
-            if (lane_ok) {
-              mbar_arrive_expect_tx(&full[s], row_bytes);
-              bulk_load_1d_hint(ring + (size_t)s * slot_bytes, H + (size_t)(im.vis_start + mtab[ui][lane]) * im.ldH, row_bytes, &full[s], once);
-            }
-          }
-          ok = __all_sync(0xffffffffu, lane_ok);
-          it_p += nm;
-        }
-        if (!ok && lane == 0) atomicExch(&abort_flag, 1);   // the copies in flight land within the consumers' bounded waits
-      }
-    } else {
-      // ---------------- consumers ----------------
-      const int cw = w - 1;
-      const int ct = cw * 32 + lane;               // consumer thread: owns the 8-column groups ct, ct + 256, ...
-      for (int ui = 0; ok && ui < nu; ++ui) {
-        const int c = meta[ui][0], k = meta[ui][1], nch = meta[ui][2], size = meta[ui][3], nm = meta[ui][4],
-                  dst = meta[ui][5], ptok = meta[ui][6];
-        float acc[kMrgVpl][8];
+    float acc[VPL][8];
 #pragma unroll
-        for (int v = 0; v < kMrgVpl; ++v)
+    for (int v = 0; v < VPL; ++v)
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[v][e] = 0.f;
+#pragma unroll 1
+    for (int mi = 0; mi < nm; mi += kMrgRows) {
+      Raw8<T> x[kMrgRows][VPL];
+#pragma unroll
+      for (int r = 0; r < kMrgRows; ++r) {
+        if (mi + r < nm) {
+          const T *row = H + (size_t)(im.vis_start + members[mi + r]) * im.ldH;
+#pragma unroll
+          for (int v = 0; v < VPL; ++v) {
+            const int g = t + v * kMrgThreads;
+            if (g < ng) x[r][v].load(row + g * 8);
+          }
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < kMrgRows; ++r) {
+        if (mi + r < nm) {
+#pragma unroll
+          for (int v = 0; v < VPL; ++v) {
+            const int g = t + v * kMrgThreads;
+            if (g < ng) x[r][v].add_to(acc[v]);
+          }
+        }
+      }
+    }
+    const float fs = center_only ? 1.0f : (float)size;
+    if (nch > 1) {
+      // scratch rows: the clusters that are summed in several chunks take theirs in cluster order
+      int base = 0;
+      for (int cc = lane; cc < c; cc += 32) {
+        const int n = chunk_off[cc + 1] - chunk_off[cc];
+        base += n > 1 ? n : 0;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) base += __shfl_xor_sync(0xffffffffu, base, o);
+      float *part = im.mpart + (size_t)(base + k) * d;
+#pragma unroll
+      for (int v = 0; v < VPL; ++v) {
+        const int g = t + v * kMrgThreads;
+        if (g < ng) {
+          reinterpret_cast<float4 *>(part + g * 8)[0] = make_float4(acc[v][0], acc[v][1], acc[v][2], acc[v][3]);
+          reinterpret_cast<float4 *>(part + g * 8)[1] = make_float4(acc[v][4], acc[v][5], acc[v][6], acc[v][7]);
+        }
+      }
+      __threadfence();
+      __syncthreads();
+      if (t == 0) s_last = (atomicAdd(&im.cticket[c], 1) == nch - 1);
+      __syncthreads();
+      if (!s_last) { u = s_next; continue; }       // the loop head synchronises before s_last and s_next are rewritten
+      __threadfence();
+      const float *p0 = im.mpart + (size_t)base * d;
+#pragma unroll
+      for (int v = 0; v < VPL; ++v) {
+        const int g = t + v * kMrgThreads;
+        if (g < ng) {
 #pragma unroll
           for (int e = 0; e < 8; ++e) acc[v][e] = 0.f;
-        for (int r = 0; r < nm; ++r, ++it_c) {
-          const int s = it_c % stages;
-          if (!mbar_wait_warp(&full[s], (it_c / stages) & 1)) { ok = false; break; }
-          const T *row = reinterpret_cast<const T *>(ring + (size_t)s * slot_bytes);
-#pragma unroll
-          for (int v = 0; v < kMrgVpl; ++v) {
-            const int g = ct + v * (kMrgConsumers * 32);
-            if (g < ng) {
-              float x[8];
-              load8<T>(row + g * 8, x);
-#pragma unroll
-              for (int e = 0; e < 8; ++e) acc[v][e] += x[e];
-            }
+          for (int kk = 0; kk < nch; ++kk) {
+            const float4 a = ld_cg_f4(p0 + (size_t)kk * d + g * 8), bq = ld_cg_f4(p0 + (size_t)kk * d + g * 8 + 4);
+            acc[v][0] += a.x; acc[v][1] += a.y; acc[v][2] += a.z; acc[v][3] += a.w;
+            acc[v][4] += bq.x; acc[v][5] += bq.y; acc[v][6] += bq.z; acc[v][7] += bq.w;
           }
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&empty[s]);
-        }
-        if (!ok) break;
-        const float fs = center_only ? 1.0f : (float)size;
-        if (nch > 1) {
-          // scratch rows: the clusters that are summed in several chunks take theirs in cluster order
-          int base = 0;
-          for (int cc = lane; cc < c; cc += 32) {
-            const int n = chunk_off[cc + 1] - chunk_off[cc];
-            base += n > 1 ? n : 0;
-          }
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) base += __shfl_xor_sync(0xffffffffu, base, o);
-          float *part = im.mpart + (size_t)(base + k) * d;
-#pragma unroll
-          for (int v = 0; v < kMrgVpl; ++v) {
-            const int g = ct + v * (kMrgConsumers * 32);
-            if (g < ng) {
-              reinterpret_cast<float4 *>(part + g * 8)[0] = make_float4(acc[v][0], acc[v][1], acc[v][2], acc[v][3]);
-              reinterpret_cast<float4 *>(part + g * 8)[1] = make_float4(acc[v][4], acc[v][5], acc[v][6], acc[v][7]);
-            }
-          }
-          __threadfence();
-          consumer_bar();
-          if (ct == 0) s_last = (atomicAdd(&im.cticket[c], 1) == nch - 1);
-          consumer_bar();
-          const bool last = s_last != 0;
-          consumer_bar();                          // s_last is read before the next unit may overwrite it
-          if (!last) continue;
-          __threadfence();
-          const float *p0 = im.mpart + (size_t)base * d;
-#pragma unroll
-          for (int v = 0; v < kMrgVpl; ++v) {
-            const int g = ct + v * (kMrgConsumers * 32);
-            if (g < ng) {
-#pragma unroll
-              for (int e = 0; e < 8; ++e) acc[v][e] = 0.f;
-              for (int kk = 0; kk < nch; ++kk) {
-                const float4 a = ld_cg_f4(p0 + (size_t)kk * d + g * 8), bq = ld_cg_f4(p0 + (size_t)kk * d + g * 8 + 4);
-                acc[v][0] += a.x; acc[v][1] += a.y; acc[v][2] += a.z; acc[v][3] += a.w;
-                acc[v][4] += bq.x; acc[v][5] += bq.y; acc[v][6] += bq.z; acc[v][7] += bq.w;
-              }
-            }
-          }
-          if (ct == 0) im.cticket[c] = 0;
-        }
-#pragma unroll
-        for (int v = 0; v < kMrgVpl; ++v) {
-          const int g = ct + v * (kMrgConsumers * 32);
-          if (g < ng) {
-            float y[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) y[e] = acc[v][e] / fs;
-            store_vec8<O>(Ho + (size_t)dst * im.ldHo + g * 8, y);
-          }
-        }
-        if (ct == 0) {
-          im.P_out[dst] = im.P[ptok];
-          im.size_out[dst] = size;
         }
       }
-      if (!ok) atomicExch(&abort_flag, 1);
+      if (t == 0) im.cticket[c] = 0;
     }
-    __syncthreads();                               // the tables are rewritten in the next round
-    if (abort_flag) break;
+#pragma unroll
+    for (int v = 0; v < VPL; ++v) {
+      const int g = t + v * kMrgThreads;
+      if (g < ng) {
+        float y[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) y[e] = acc[v][e] / fs;
+        store_vec8<O>(Ho + (size_t)dst * im.ldHo + g * 8, y);
+      }
+    }
+    if (t == 0) {
+      im.P_out[dst] = im.P[ptok];
+      im.size_out[dst] = size;
+    }
+    u = s_next;
   }
-  __syncthreads();
-  if (t == 0 && abort_flag) atomicMin(&im.cnt[PACT_CNT_STATUS], (int)PACT_ERR_TIMEOUT);
 }
 
 void launch_lists(const Batch &bt, int maxN, cudaStream_t st) {
@@ -386,15 +337,20 @@ static size_t g_merge_smem_max = 48 * 1024;
 
 template <typename T, typename O>
 static cudaError_t launch_merge_t(const Batch &bt, int maxN, const ClusterCfg &cfg, cudaStream_t st) {
-  const size_t off = (((size_t)maxN + 2) * sizeof(int) + 127) / 128 * 128;
-  const size_t slot = ((size_t)bt.d * sizeof(T) + 127) / 128 * 128;
-  if (off + 2 * slot > g_merge_smem_max) return cudaErrorInvalidConfiguration;
-  int stages = (int)((g_merge_smem_max - off) / slot);
-  if (stages > kMrgStagesMax) stages = kMrgStagesMax;
-  int X = cfg.sm_count / bt.B;
+  const size_t smem = ((size_t)maxN + 2) * sizeof(int);
+  if (smem > g_merge_smem_max) return cudaErrorInvalidConfiguration;
+  int X = 3 * cfg.sm_count / bt.B;
   if (X < 1) X = 1;
-  k_merge<T, O><<<dim3(X, bt.B), kMrgThreads, off + (size_t)stages * slot, st>>>(bt, stages, (int)slot, (int)off);
+  dim3 grid(X, bt.B);
+  if (bt.d <= kMrgThreads * 2 * 8) k_merge<T, O, 2><<<grid, kMrgThreads, smem, st>>>(bt);
+  else k_merge<T, O, kMrgVpl><<<grid, kMrgThreads, smem, st>>>(bt);
   return cudaGetLastError();
+}
+
+template <typename T, typename O> static cudaError_t merge_attr(int v) {
+  cudaError_t e = cudaFuncSetAttribute(k_merge<T, O, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, v);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(k_merge<T, O, kMrgVpl>, cudaFuncAttributeMaxDynamicSharedMemorySize, v);
 }
 
 cudaError_t merge_configure() {
@@ -403,20 +359,19 @@ cudaError_t merge_configure() {
   if (e != cudaSuccess) return e;
   e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
   if (e != cudaSuccess) return e;
-  g_merge_smem_max = (size_t)optin - 5120;       // the kernel also has about 4 KB of static shared memory
+  g_merge_smem_max = (size_t)optin - 2048;
   const int v = (int)g_merge_smem_max;
-  e = cudaFuncSetAttribute(k_merge<__nv_bfloat16, __nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, v);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_merge<__nv_bfloat16, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, v);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_merge<float, __nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, v);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_merge<float, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, v);
+  e = merge_attr<__nv_bfloat16, __nv_bfloat16>(v);
+  if (e == cudaSuccess) e = merge_attr<__nv_bfloat16, float>(v);
+  if (e == cudaSuccess) e = merge_attr<float, __nv_bfloat16>(v);
+  if (e == cudaSuccess) e = merge_attr<float, float>(v);
   return e;
 }
 
-// largest N the merge kernel takes: its chunk offsets and at least two ring slots live in shared memory
+// largest N the merge kernel takes: its chunk offsets live in shared memory
 int merge_max_tokens(int d, int elt) {
-  const size_t slot = ((size_t)d * elt + 127) / 128 * 128;
-  if (g_merge_smem_max < 2 * slot + 256) return 0;
-  return (int)((g_merge_smem_max - 2 * slot - 128) / sizeof(int)) - 2;
+  (void)d; (void)elt;
+  return (int)(g_merge_smem_max / sizeof(int)) - 2;
 }
 
 cudaError_t launch_merge(const Batch &bt, int maxN, bool in_bf16, bool out_bf16, const ClusterCfg &cfg, cudaStream_t st) {
