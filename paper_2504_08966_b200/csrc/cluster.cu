@@ -348,6 +348,7 @@ __global__ void __launch_bounds__(256) k_centers(const __grid_constant__ Batch b
         pending = 1;
       }
     }
+    if (pending) __nanosleep(100);                 // the masks are polled by thousands of warps: do not hammer them
   }
   if (lane == 0 && total > 0) {
     for (int b = 0; b < bt.B; ++b) {
@@ -361,52 +362,97 @@ __global__ void __launch_bounds__(256) k_centers(const __grid_constant__ Batch b
   __threadfence();
   grid.sync();
   TL_POINT(bt.img[0], 12);
-  for (int item = gw; item < total; item += nwarps) {
-    int b = 0;
-    while (item >= qs[b + 1]) ++b;
+  // Cluster id of a centre = number of centres with a lower index.  The centre mask of an image is read
+  // once per CTA into shared memory with its running bit counts (every warp reading the same few words
+  // from global memory makes them a hot spot); images too large for the staging buffer take the words
+  // from global memory.
+  __shared__ int wsum3[8];
+  __shared__ int s_carry3;
+  for (int b = 0; b < bt.B; ++b) {
     const ImgDesc &im = bt.img[b];
-    const int r = item - qs[b], q = qs[b + 1] - qs[b], nw = (q + 31) >> 5;
-    // this lane's words of the centre mask, its share of the row and the row's bookkeeping: one round trip
-    int below = 0, all = 0;
-    uint32_t myword = 0u;
-    for (int wd = lane; wd < nw; wd += 32) {
-      const uint32_t m = __ldcg(&im.cmask[wd]);
-      const int pc = __popc(m);
-      all += pc;
-      if (wd < (r >> 5)) below += pc;
-      else if (wd == (r >> 5)) { below += __popc(m & ((1u << (r & 31)) - 1u)); myword = m; }
-    }
-    const T *src = reinterpret_cast<const T *>(im.Kp) + (size_t)r * bt.d_k;
-    const int nv = bt.d_k / V;
-    uint4 buf[4];
+    const int q = qs[b + 1] - qs[b], nw = (q + 31) >> 5;
+    const bool staged = q <= keys_cap;              // nw words and nw counts fit where the densities were
+    uint32_t *cm = reinterpret_cast<uint32_t *>(skeys);
+    int *pref = reinterpret_cast<int *>(skeys) + nw;
+    __syncthreads();
+    if (staged) {
+      if (threadIdx.x == 0) s_carry3 = 0;
+      __syncthreads();
+      for (int base = 0; base < nw; base += 256) {
+        const int wd = base + threadIdx.x;
+        const uint32_t m = wd < nw ? __ldcg(&im.cmask[wd]) : 0u;
+        const int pc = __popc(m);
+        int x = pc;
 #pragma unroll
-    for (int u = 0; u < 4; ++u)
-      if (lane + 32 * u < nv) buf[u] = __ldcg(reinterpret_cast<const uint4 *>(src) + lane + 32 * u);
-    const int tok = im.kept_idx[r];
-    const auto rnr = rn_kept<D>(im)[r];
+        for (int o = 1; o < 32; o <<= 1) {
+          const int y = __shfl_up_sync(0xffffffffu, x, o);
+          if (lane >= o) x += y;
+        }
+        if (lane == 31) wsum3[threadIdx.x >> 5] = x;
+        __syncthreads();
+        int off = s_carry3;
+        for (int k = 0; k < (int)(threadIdx.x >> 5); ++k) off += wsum3[k];
+        if (wd < nw) { cm[wd] = m; pref[wd] = off + x - pc; }
+        __syncthreads();
+        if (threadIdx.x == 255) s_carry3 = off + x;
+        __syncthreads();
+      }
+    }
+    int item = gw;
+    if (item < qs[b]) item += ((qs[b] - item + nwarps - 1) / nwarps) * nwarps;
+    for (; item < qs[b + 1]; item += nwarps) {
+      const int r = item - qs[b];
+      int c, all;
+      bool is_center;
+      if (staged) {
+        const uint32_t m = cm[r >> 5];
+        is_center = ((m >> (r & 31)) & 1u) != 0u;
+        c = pref[r >> 5] + __popc(m & ((1u << (r & 31)) - 1u));
+        all = s_carry3;
+      } else {
+        int below = 0;
+        all = 0;
+        uint32_t myword = 0u;
+        for (int wd = lane; wd < nw; wd += 32) {
+          const uint32_t m = __ldcg(&im.cmask[wd]);
+          const int pc = __popc(m);
+          all += pc;
+          if (wd < (r >> 5)) below += pc;
+          else if (wd == (r >> 5)) { below += __popc(m & ((1u << (r & 31)) - 1u)); myword = m; }
+        }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      below += __shfl_xor_sync(0xffffffffu, below, o);
-      all += __shfl_xor_sync(0xffffffffu, all, o);
-      myword |= __shfl_xor_sync(0xffffffffu, myword, o);
-    }
-    if (r == 0 && lane == 0) {
-      im.cnt[PACT_CNT_C] = all;
-      if (im.C_user) *im.C_user = all;
-    }
-    if (!((myword >> (r & 31)) & 1u)) continue;
-    const int c = below;
-    if (lane == 0) {
-      im.cid[r] = c;
-      im.center_idx[c] = tok;
-      if (im.center_idx_user) im.center_idx_user[c] = tok;
-      rn_cen<D>(im)[c] = rnr;
-    }
-    uint4 *dst = reinterpret_cast<uint4 *>(reinterpret_cast<T *>(im.Kcen) + (size_t)c * bt.d_k);
+        for (int o = 16; o > 0; o >>= 1) {
+          below += __shfl_xor_sync(0xffffffffu, below, o);
+          all += __shfl_xor_sync(0xffffffffu, all, o);
+          myword |= __shfl_xor_sync(0xffffffffu, myword, o);
+        }
+        c = below;
+        is_center = ((myword >> (r & 31)) & 1u) != 0u;
+      }
+      if (r == 0 && lane == 0) {
+        im.cnt[PACT_CNT_C] = all;
+        if (im.C_user) *im.C_user = all;
+      }
+      if (!is_center) continue;
+      const T *src = reinterpret_cast<const T *>(im.Kp) + (size_t)r * bt.d_k;
+      const int nv = bt.d_k / V;
+      uint4 buf[4];
 #pragma unroll
-    for (int u = 0; u < 4; ++u)
-      if (lane + 32 * u < nv) dst[lane + 32 * u] = buf[u];
-    for (int v = lane + 128; v < nv; v += 32) dst[v] = __ldcg(reinterpret_cast<const uint4 *>(src) + v);
+      for (int u = 0; u < 4; ++u)
+        if (lane + 32 * u < nv) buf[u] = __ldcg(reinterpret_cast<const uint4 *>(src) + lane + 32 * u);
+      if (lane == 0) {
+        const int tok = im.kept_idx[r];
+        im.cid[r] = c;
+        im.center_idx[c] = tok;
+        if (im.center_idx_user) im.center_idx_user[c] = tok;
+        rn_cen<D>(im)[c] = rn_kept<D>(im)[r];
+      }
+      uint4 *dst = reinterpret_cast<uint4 *>(reinterpret_cast<T *>(im.Kcen) + (size_t)c * bt.d_k);
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (lane + 32 * u < nv) dst[lane + 32 * u] = buf[u];
+      for (int v = lane + 128; v < nv; v += 32) dst[v] = __ldcg(reinterpret_cast<const uint4 *>(src) + v);
+    }
   }
 }
 
