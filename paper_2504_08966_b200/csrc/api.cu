@@ -9,7 +9,7 @@
 
 using namespace pact;
 
-constexpr int kProfStages = 10;
+constexpr int kProfStages = 9;
 
 struct pact_ctx {
   int d, n_qh, n_kvh, d_h, d_k, n_qcols;
@@ -32,7 +32,7 @@ struct pact_graph {
 };
 
 static const char *const kStageNames[kProfStages] = {
-    "prepass", "logits", "scores", "select_gather", "gram_density", "centers", "assign", "label", "lists",
+    "prepass", "logits", "scores", "select_gather", "gram_density", "centers", "assign", "label_lists",
     "merge"};
 
 namespace {
@@ -447,7 +447,7 @@ pact_status pact_merge(pact_ctx *ctx, const pact_image *img, const int32_t *labe
   CK(cudaMemsetAsync(m.cnt, 0, 32 * sizeof(int32_t), st));
   CK(cudaMemsetAsync(m.csize, 0, (size_t)m.Np * sizeof(int32_t), st));
   CK(cudaMemsetAsync(m.cticket, 0, (size_t)m.Np * sizeof(int32_t), st));
-  launch_lists(bt, img->N, st);
+  launch_lists(bt, img->N, ctx->in == PACT_BF16, false, st);
   CK(launch_merge(bt, img->N, ctx->in == PACT_BF16, ctx->out == PACT_BF16, ctx->ccfg, st));
   ctx->launches += 2;
   CK(cudaGetLastError());
@@ -509,10 +509,9 @@ pact_status pact_reduce(pact_ctx *ctx, const pact_image *imgs, int B, const pact
     if (ctx->umma) CK(launch_assign_umma(bt, cmaxN, false, ctx->ccfg, st));
     else launch_assign(bt, cmaxN, bf, ROWS_ALL, ctx->ccfg, st);
     CK(mark());
-    launch_label(bt, cmaxN, bf, ROWS_ALL, st);      CK(mark());
-    launch_lists(bt, cmaxN, st);                    CK(mark());
+    launch_lists(bt, cmaxN, bf, true, st);          CK(mark());
     CK(launch_merge(bt, cmaxN, bf, ctx->out == PACT_BF16, ctx->ccfg, st));  CK(mark());
-    ctx->launches += 10;
+    ctx->launches += 9;
     CK(cudaGetLastError());
     for (int b = 0; b < nb; ++b)
       CK(cudaMemcpyAsync(bt.img[b].counters_user, bt.img[b].cnt, PACT_N_COUNTERS * sizeof(int32_t),

@@ -42,8 +42,9 @@ cudaError_t launch_gram_umma(const Batch &bt, int maxN, const ClusterCfg &cfg, c
 cudaError_t launch_assign_umma(const Batch &bt, int maxN, bool kept_rows, const ClusterCfg &cfg, cudaStream_t st);
 
 // merge.cu
-// member lists from label[]; csize and cticket must be zero
-void launch_lists(const Batch &bt, int maxN, cudaStream_t st);
+// member lists from label[] (from_best: labels are first formed from the nearest-centre pass, all tokens);
+// csize and cticket must be zero
+void launch_lists(const Batch &bt, int maxN, bool bf16, bool from_best, cudaStream_t st);
 cudaError_t launch_merge(const Batch &bt, int maxN, bool in_bf16, bool out_bf16, const ClusterCfg &cfg, cudaStream_t st);
 cudaError_t merge_configure();
 int merge_max_tokens(int d, int elt);      // largest N the merge kernel takes (its chunk offsets live in shared memory)

@@ -81,7 +81,12 @@ __device__ __forceinline__ float4 ld_cg_f4(const float *p) {
 // below c, for c = 0..C.  The members of cluster c are then, in ascending token order, the entries
 // [bstart[b][c], bstart[b][c+1]) of blocklist[b] for b = 0, 1, ...  Cluster sizes are added up with
 // integer atomics.
+// FROM_BEST: the labels are first formed here from the nearest-centre pass (survivors: cluster id of the
+// nearest centre, a centre its own id; pruned tokens: that id iff the distance is strictly below
+// alpha * d_c, else -1) and written out; otherwise label[] is given.
+template <typename T, bool FROM_BEST>
 __global__ void __launch_bounds__(kListBlock) k_lists(const __grid_constant__ Batch bt) {
+  using D = typename DistOf<T>::type;
   const ImgDesc &im = bt.img[blockIdx.y];
   TL_SCOPE(im, 8);
   const int N = im.N;
@@ -90,7 +95,37 @@ __global__ void __launch_bounds__(kListBlock) k_lists(const __grid_constant__ Ba
   if (b >= nblk) return;
   __shared__ int slab[kListBlock], sorted_lab[kListBlock];
   const int i = b * kListBlock + t;
-  const int lab = i < N ? im.label[i] : -1;
+  int lab = -1;
+  if (FROM_BEST) {
+    int joined = 0, dropped = 0, band = 0;
+    if (i < N) {
+      const int r = im.slot[i];                     // >= 0: survivor position; < 0: pruned
+      const unsigned long long pk = im.best[i];
+      lab = (int)(pk & 0xFFFFFFFFull);
+      const float dd = __uint_as_float((uint32_t)(pk >> 32));
+      if (r >= 0) {
+        if ((im.cmask[r >> 5] >> (r & 31)) & 1u) lab = im.cid[r];
+      } else {
+        if (D::in_band_t(dd, im)) ++band;
+        if (D::below_t(dd, im)) ++joined; else { lab = -1; ++dropped; }
+      }
+      im.label[i] = lab;
+      if (im.label_user) im.label_user[i] = lab;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      joined += __shfl_xor_sync(0xffffffffu, joined, o);
+      dropped += __shfl_xor_sync(0xffffffffu, dropped, o);
+      band += __shfl_xor_sync(0xffffffffu, band, o);
+    }
+    if ((t & 31) == 0) {
+      if (joined) atomicAdd(&im.cnt[PACT_CNT_R], joined);
+      if (dropped) atomicAdd(&im.cnt[PACT_CNT_DISCARDED], dropped);
+      if (band) atomicAdd(&im.cnt[PACT_CNT_BAND_ADC], band);
+    }
+  } else {
+    lab = i < N ? im.label[i] : -1;
+  }
   const int C = *im.C_ptr;
   const int key = lab < 0 ? 0x7fffffff : lab;
   slab[t] = key;
@@ -329,8 +364,14 @@ k_merge(const __grid_constant__ Batch bt) {
   }
 }
 
-void launch_lists(const Batch &bt, int maxN, cudaStream_t st) {
-  k_lists<<<dim3((maxN + kListBlock - 1) / kListBlock, bt.B), kListBlock, 0, st>>>(bt);
+void launch_lists(const Batch &bt, int maxN, bool bf16, bool from_best, cudaStream_t st) {
+  const dim3 grid((maxN + kListBlock - 1) / kListBlock, bt.B);
+  if (from_best) {
+    if (bf16) k_lists<__nv_bfloat16, true><<<grid, kListBlock, 0, st>>>(bt);
+    else k_lists<float, true><<<grid, kListBlock, 0, st>>>(bt);
+  } else {
+    k_lists<float, false><<<grid, kListBlock, 0, st>>>(bt);
+  }
 }
 
 static size_t g_merge_smem_max = 48 * 1024;
