@@ -28,6 +28,9 @@ sys.path.insert(0, ROOT)
 METRIC = "visual tokens reduced/sec and per-image latency (us) at N=7290; % of roofline"
 UNIT = "tokens/s"
 N_COPIES = 4          # input copies rotated between steps so that no step finds its inputs in L2
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
+# (workload, kernel) -> bytes; absent = not captured for the kernel as it stands
+NCU_TRAFFIC: dict = {}
 
 
 def _peaks():
@@ -264,10 +267,11 @@ def main():
     t_hbm = per_img_bytes / (pk["hbm_gbs"] * 1e9)
     t_tc = per_img_flops / (pk["bf16_tflops"] * 1e12)
     t_roof = max(t_hbm, t_tc) * B
+    n_qcols = wl.n_qh * wl.d_h
     alg = {   # algorithmic bytes (hbm) or flops (tensor) of one launch of each kernel, image 0 scaled by B
-        "qsum": ("hbm", img0.N * wl.n_qh * wl.d_h * 2.0),
-        "logit_norm": ("hbm", img0.N * d * 2.0 + img0.N * d_k * 2.0),
-        "keynorm_gather": ("hbm", img0.N * d_k * 2.0 + q * d_k * 2.0),
+        "prepass": ("hbm", img0.N * d * 2.0 + img0.N * d_k * 2.0 + img0.N * n_qcols * 2.0),
+        "logits": ("hbm", img0.N * d_k * 2.0 + img0.N * wl.n_qh * 8.0),
+        "select_gather": ("hbm", 2.0 * q * d_k * 2.0 + img0.N * 4.0),
         "gram_density": ("tensor", 2.0 * d_k * (q * (q + 1) / 2)),
         "assign": ("tensor", 2.0 * d_k * img0.N * Cn),
         "merge": ("hbm", (q + r) * d * 2.0 + Cn * d * 2.0 + 2 * T * d * 2.0),
@@ -283,7 +287,7 @@ def main():
         else:
             ach, peak, unit = amount / secs / 1e12, pk["bf16_tflops"], "TFLOP/s"
         roof = {"kernel": top, "bound": kind, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
-                "traffic": None, "peak_source": pk["source"], "launch_us": stages_us[top]}
+                "traffic": NCU_TRAFFIC.get((wl.name, top)), "peak_source": pk["source"], "launch_us": stages_us[top]}
     elif top is not None:
         roof = {"kernel": top, "bound": "latency", "achieved": None, "peak": None, "unit": None, "frac": None,
                 "traffic": None, "launch_us": stages_us[top],
