@@ -30,7 +30,12 @@ UNIT = "tokens/s"
 N_COPIES = 4          # input copies rotated between steps so that no step finds its inputs in L2
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
 # (workload, kernel) -> bytes; absent = not captured for the kernel as it stands
-NCU_TRAFFIC: dict = {}
+NCU_TRAFFIC: dict = {
+    ("single_image", "merge"): 52311808 + 444160,
+    ("single_image", "prepass"): 67237376 + 438784,
+    ("single_image", "gram_density"): 4024064,
+    ("single_image", "assign"): 8372224,
+}
 
 
 def _peaks():

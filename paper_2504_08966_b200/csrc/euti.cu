@@ -73,13 +73,12 @@ __global__ void __launch_bounds__(kPreThreads) k_prepass(const __grid_constant__
         const T *Kc = reinterpret_cast<const T *>(im.Kc);
         int i = 0;
         bool ok = true;
-        const uint64_t keep = l2_policy_evict_last();   // the merge reads the hidden-state rows again
         for (; i < ntok; ++i) {
           const int s = i % stages;
           if (!mbar_wait(&empty[s], ((i / stages) & 1) ^ 1)) { ok = false; break; }
           unsigned char *dst = ring + (size_t)s * slot_bytes;
           mbar_arrive_expect_tx(&full[s], hbytes + kbytes);
-          if (want_h) bulk_load_1d_hint(dst, H + (size_t)(im.vis_start + t0 + i) * im.ldH, hbytes, &full[s], keep);
+          if (want_h) bulk_load_1d(dst, H + (size_t)(im.vis_start + t0 + i) * im.ldH, hbytes, &full[s]);
           if (want_k) bulk_load_1d(dst + hbytes, Kc + (size_t)(t0 + i) * im.ldKc, kbytes, &full[s]);
         }
         if (!ok) {

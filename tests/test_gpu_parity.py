@@ -157,6 +157,32 @@ def test_bitwise_deterministic_run_to_run():
     assert np.array_equal(a[0]["score"].view(np.int32), b[0]["score"].view(np.int32))
 
 
+def test_more_than_16384_tokens_takes_the_general_select_path():
+    """Beyond 16384 tokens the split keeps its keys in shared memory instead of registers."""
+    wl = workloads.single_image(seed=75, N=17011, T=5, n_blobs=60, lam=0.85, d=128, n_h=2, d_h=32)
+    outs = _check_workload(wl, torch.float32)
+    assert outs[0]["q"] >= 2551
+
+
+@pytest.mark.parametrize("N", [40000, 60001])
+def test_stage_prune_large_inputs(N):
+    """40000 keys fit in shared memory, 60001 are re-read from the scores."""
+    from paper_2504_08966_b200 import binding as pb
+    ctx = pb.Context(256, 2, 2, 32, torch.bfloat16, torch.bfloat16)
+    g = torch.Generator().manual_seed(N)
+    s32 = (torch.rand(N, generator=g) * torch.exp(4 * torch.randn(N, generator=g))).numpy().astype(np.float32)
+    s32[7] = s32[N - 3] = s32[N // 2]
+    for lam in (0.37, 0.9):
+        tau, keep, kept, pruned = orc.split(s32, lam)
+        dev = lambda dt: torch.empty(N, dtype=dt, device="cuda")
+        keep_d, kept_d, pruned_d, counts = dev(torch.uint8), dev(torch.int32), dev(torch.int32), torch.zeros(2, dtype=torch.int32, device="cuda")
+        ctx.pact_prune(torch.from_numpy(s32).cuda(), pb.make_params(lam=lam), keep_d, kept_d, pruned_d, counts)
+        q, m = counts.cpu().tolist()
+        assert q == kept.size and m == pruned.size
+        assert np.array_equal(keep_d.cpu().numpy().astype(bool), keep)
+        assert np.array_equal(kept_d[:q].cpu().numpy(), kept) and np.array_equal(pruned_d[:m].cpu().numpy(), pruned)
+
+
 def test_graph_replay_matches_direct_call_bitwise():
     from paper_2504_08966_b200 import binding as pb
     wl = workloads.single_image(seed=72, N=2100, T=10, n_blobs=50)
