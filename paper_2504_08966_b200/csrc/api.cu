@@ -240,7 +240,7 @@ pact_status pact_create(pact_ctx **out, int d, int n_qh, int n_kvh, int d_h, pac
     e = cudaGetDeviceProperties(&pr, c->device);
     if (e == cudaSuccess && pr.major != 10) { delete c; return PACT_ERR_UNSUPPORTED; }
   }
-  if (e == cudaSuccess) e = euti_configure(c->n_qcols, c->n_qh, c->d, c->d_k, c->elt);
+  if (e == cudaSuccess) e = euti_configure(c->n_qcols, c->n_qh);
   if (e == cudaSuccess) e = cluster_configure(&c->ccfg);
   if (e == cudaSuccess) e = merge_configure();
   if (e == cudaSuccess && in == PACT_BF16) e = umma_configure();

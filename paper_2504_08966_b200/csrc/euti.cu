@@ -4,7 +4,7 @@
 // rare double-rounding cases.
 //
 //   k_prepass        one pass over Q, H and the clustering keys: column sums of Q -> global query,
-//                    hidden-state norms, inverse key norms (HBM-bound, the only full read of H)
+//                    hidden-state norms, inverse key norms (HBM-bound, the first of two reads of H)
 //   k_logits         k_i . Qglobal per head, CTA-local softmax pieces (max, sum of exp)
 //   k_scores         merges the pieces, writes the float32 scores
 //   k_select_gather  every CTA selects the threshold and compacts (identical results in every CTA),
@@ -13,7 +13,6 @@
 // The kernels are short chains of dependent memory round trips; each issues all the loads it can
 // before it consumes the first.
 #include "kernels.cuh"
-#include "tma.cuh"
 
 namespace pact {
 
@@ -23,22 +22,20 @@ __device__ __forceinline__ double ld_cg_f64(const double *p) {
   return v;
 }
 
-constexpr int kPreConsumers = 8;                           // warps that reduce rows
-constexpr int kPreThreads = 32 * (1 + kPreConsumers);      // warp 0 issues the bulk copies
-constexpr int kPreStagesMax = 16;
-constexpr int kQCtasMax = kQPartRows;                      // CTAs that reduce Q
+constexpr int kPreThreads = 512;
+constexpr int kTokWarps = kPreThreads / 32;   // tokens per CTA of the token part of k_prepass
+constexpr int kQCtasMax = kQPartRows;         // CTAs that reduce Q
 
 // ---- Eq. 1 and the norms -----------------------------------------------------------------------
-// grid (GQ + X, B), 288 threads.
+// grid (GQ + ceil(maxN / 16), B), 512 threads.
 //  CTAs [0, GQ): column sums of a contiguous block of rows of Q; the last of them to finish adds
 //                the GQ partial sums in index order and writes the global query.
-//  other CTAs:   persistent, one per SM: CTA x takes a contiguous block of visual tokens.  Warp 0
-//                streams each token's hidden-state row and clustering-key row into a ring of shared
-//                memory slots with bulk copies (a steady depth of `stages` rows in flight per SM);
-//                warps 1-8 take the slots in turn: |h_i| (double) and 1 / |k_i|.
+//  other CTAs:   one warp per visual token; every 16-byte load of the token's clustering-key row and
+//                hidden-state row is issued before the first is used: |h_i| (double) and 1 / |k_i|.
+// (A variant that streamed the rows through a shared-memory ring with bulk copies measured the same on
+// one image and worse on batches: bulk copies issued row by row complete at about 20 GB/s per SM.)
 template <typename T>
-__global__ void __launch_bounds__(kPreThreads) k_prepass(const __grid_constant__ Batch bt, int GQ, int stages,
-                                                          int slot_bytes) {
+__global__ void __launch_bounds__(kPreThreads) k_prepass(const __grid_constant__ Batch bt, int GQ) {
   using D = typename DistOf<T>::type;
   using rn_t = typename D::rn_t;
   constexpr int V = Vec<T>::N;
@@ -46,75 +43,32 @@ __global__ void __launch_bounds__(kPreThreads) k_prepass(const __grid_constant__
   TL_SCOPE(im, 0);
   const int t = threadIdx.x, lane = t & 31, w = t >> 5;
   if ((int)blockIdx.x >= GQ) {
-    extern __shared__ __align__(128) unsigned char ring[];
-    __shared__ uint64_t full[kPreStagesMax], empty[kPreStagesMax];
-    __shared__ int abort_flag;
-    const int X = gridDim.x - GQ, x = blockIdx.x - GQ;
-    const int per = (im.N + X - 1) / X;
-    const int t0 = min(im.N, x * per), ntok = min(im.N, t0 + per) - t0;
-    const bool want_h = im.H && !(im.flags & PACT_FLAG_NO_NORM);
-    const bool want_k = im.Kc != nullptr;
-    const uint32_t hbytes = want_h ? (uint32_t)bt.d * sizeof(T) : 0u;
-    const uint32_t kbytes = want_k ? (uint32_t)bt.d_k * sizeof(T) : 0u;
-    if (ntok <= 0) return;
-    if (hbytes + kbytes == 0u) {                     // nothing to read: the norm factor is switched off
-      for (int i = t; i < ntok; i += kPreThreads) if (im.H) im.nrm[t0 + i] = 1.0;
-      return;
-    }
-    if (t == 0) {
-      for (int s = 0; s < stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-      abort_flag = 0;
-      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    __syncthreads();
-    if (w == 0) {
-      if (lane == 0) {
-        const T *H = reinterpret_cast<const T *>(im.H);
-        const T *Kc = reinterpret_cast<const T *>(im.Kc);
-        int i = 0;
-        bool ok = true;
-        for (; i < ntok; ++i) {
-          const int s = i % stages;
-          if (!mbar_wait(&empty[s], ((i / stages) & 1) ^ 1)) { ok = false; break; }
-          unsigned char *dst = ring + (size_t)s * slot_bytes;
-          mbar_arrive_expect_tx(&full[s], hbytes + kbytes);
-          if (want_h) bulk_load_1d(dst, H + (size_t)(im.vis_start + t0 + i) * im.ldH, hbytes, &full[s]);
-          if (want_k) bulk_load_1d(dst + hbytes, Kc + (size_t)(t0 + i) * im.ldKc, kbytes, &full[s]);
-        }
-        if (!ok) {
-          atomicExch(&abort_flag, 1);
-          // every copy that was issued lands before this CTA's shared memory is given up
-          const int armed = i < stages ? i : stages;
-          for (int k = 0; k < armed; ++k) {
-            const int j = i - 1 - k;
-            mbar_wait(&full[j % stages], (j / stages) & 1);
-          }
-        }
+    const int tok = ((int)blockIdx.x - GQ) * kTokWarps + w;
+    if (tok >= im.N) return;
+    constexpr int UK = 4;
+    const T *krow = im.Kc ? reinterpret_cast<const T *>(im.Kc) + (size_t)tok * im.ldKc : nullptr;
+    const int nvk = krow ? bt.d_k / V : 0;
+    uint4 kb[UK];
+#pragma unroll
+    for (int u = 0; u < UK; ++u)
+      if (lane + 32 * u < nvk) kb[u] = __ldg(reinterpret_cast<const uint4 *>(krow) + lane + 32 * u);
+    if (im.H) {
+      double nn = 1.0;
+      if (!(im.flags & PACT_FLAG_NO_NORM)) {
+        const T *hrow = reinterpret_cast<const T *>(im.H) + (size_t)(im.vis_start + tok) * im.ldH;
+        nn = sqrt(warp_sum(row_sumsq_lane<T, 16>(hrow, bt.d, lane)));
       }
-    } else {
-      const int cw = w - 1;
-      const int nvh = (int)(hbytes / 16), nvk = (int)(kbytes / 16);
-      for (int i = cw; i < ntok; i += kPreConsumers) {
-        const int s = i % stages;
-        if (!mbar_wait_warp(&full[s], (i / stages) & 1)) { atomicExch(&abort_flag, 1); break; }
-        const uint4 *src = reinterpret_cast<const uint4 *>(ring + (size_t)s * slot_bytes);
-        double acc_h = 0.0, acc_k = 0.0;
-        for (int v = lane; v < nvh; v += 32) sumsq_accumulate<T>(src[v], acc_h);
-        for (int v = lane; v < nvk; v += 32) sumsq_accumulate<T>(src[nvh + v], acc_k);
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&empty[s]);       // the slot may be refilled
-        if (im.H) {
-          const double nn = want_h ? sqrt(warp_sum(acc_h)) : 1.0;
-          if (lane == 0) im.nrm[t0 + i] = nn;
-        }
-        if (want_k) {
-          const double ss = warp_sum(acc_k);
-          if (lane == 0) rn_tok<D>(im)[t0 + i] = (rn_t)(1.0 / sqrt(fmax(ss, 1e-40)));
-        }
-      }
+      if (lane == 0) im.nrm[tok] = nn;
     }
-    __syncthreads();
-    if (t == 0 && abort_flag) atomicMin(&im.cnt[PACT_CNT_STATUS], (int)PACT_ERR_TIMEOUT);
+    if (krow) {
+      double acc = 0.0;
+#pragma unroll
+      for (int u = 0; u < UK; ++u)
+        if (lane + 32 * u < nvk) sumsq_accumulate<T>(kb[u], acc);
+      if (nvk > 32 * UK) acc += row_sumsq_lane<T, 8>(krow, bt.d_k, lane, 32 * UK);
+      const double ss = warp_sum(acc);
+      if (lane == 0) rn_tok<D>(im)[tok] = (rn_t)(1.0 / sqrt(fmax(ss, 1e-40)));
+    }
     return;
   }
   if (!im.Q) return;
@@ -122,10 +76,9 @@ __global__ void __launch_bounds__(kPreThreads) k_prepass(const __grid_constant__
   const int chunk = (im.N + GQ - 1) / GQ;
   const int r0 = min(im.N, g * chunk), r1 = min(im.N, r0 + chunk);
   const int ncolv = bt.n_qcols / V;
-  constexpr int kQThreads = 256;                     // threads of a Q CTA that take part
-  const int cpp = min(ncolv, kQThreads);             // column vectors per pass
-  const int groups = kQThreads / cpp;                // row groups per pass
-  __shared__ double sm[kQThreads * V];
+  const int cpp = min(ncolv, kPreThreads);   // column vectors per pass
+  const int groups = kPreThreads / cpp;      // row groups per pass
+  __shared__ double sm[kPreThreads * V];
   const T *Q = reinterpret_cast<const T *>(im.Q);
   const int c = t % cpp, gi = t / cpp;
   constexpr int UQ = 8;
@@ -151,10 +104,8 @@ __global__ void __launch_bounds__(kPreThreads) k_prepass(const __grid_constant__
         }
       }
     }
-    if (t < kQThreads) {
 #pragma unroll
-      for (int k = 0; k < V; ++k) sm[t * V + k] = acc[k];
-    }
+    for (int k = 0; k < V; ++k) sm[t * V + k] = acc[k];
     __syncthreads();
     if (gi == 0 && cbase + c < ncolv) {
 #pragma unroll
@@ -175,8 +126,13 @@ __global__ void __launch_bounds__(kPreThreads) k_prepass(const __grid_constant__
   __threadfence();
   for (int col = t; col < bt.n_qcols; col += kPreThreads) {
     double s = 0.0;
-#pragma unroll 8
-    for (int h = 0; h < GQ; ++h) s += ld_cg_f64(&im.qpart[(size_t)h * bt.n_qcols + col]);
+    for (int h0 = 0; h0 < GQ; h0 += 16) {            // 16 partial sums in flight, added in index order
+      double v[16];
+#pragma unroll
+      for (int u = 0; u < 16; ++u) v[u] = h0 + u < GQ ? ld_cg_f64(&im.qpart[(size_t)(h0 + u) * bt.n_qcols + col]) : 0.0;
+#pragma unroll
+      for (int u = 0; u < 16; ++u) s += v[u];
+    }
     im.qg[col] = s / (double)im.N;
   }
   if (t == 0) im.cnt[16] = 0;
@@ -570,7 +526,6 @@ __global__ void __launch_bounds__(1024) k_select_gather(const __grid_constant__ 
 namespace {
 int g_sm_count = 148;
 size_t g_smem_optin = 48 * 1024;
-size_t g_prepass_ring = 40 * 1024;           // bytes of shared memory the prepass may use for its ring
 constexpr size_t kSelectReserve = 4096;      // static shared memory of k_select_gather, rounded up
 
 int q_ctas(int maxN) {
@@ -581,20 +536,9 @@ int q_ctas(int maxN) {
 
 void launch_prepass(const Batch &bt, int maxN, bool bf16, cudaStream_t st) {
   const int GQ = q_ctas(maxN);
-  const int elt = bf16 ? 2 : 4;
-  int slot = (bt.d + bt.d_k) * elt;
-  slot = (slot + 127) / 128 * 128;
-  int stages = (int)(g_prepass_ring / (size_t)slot);
-  if (stages > kPreStagesMax) stages = kPreStagesMax;
-  if (stages < 2) stages = 2;                      // pact_create has checked that two slots fit
-  int X = g_sm_count / bt.B;
-  if (X < 1) X = 1;
-  const int cap = (maxN + 7) / 8;                  // at least 8 tokens per CTA
-  if (X > cap) X = cap;
-  dim3 grid(GQ + X, bt.B);
-  const size_t smem = (size_t)stages * slot;
-  if (bf16) k_prepass<__nv_bfloat16><<<grid, kPreThreads, smem, st>>>(bt, GQ, stages, slot);
-  else k_prepass<float><<<grid, kPreThreads, smem, st>>>(bt, GQ, stages, slot);
+  dim3 grid(GQ + (maxN + kTokWarps - 1) / kTokWarps, bt.B);
+  if (bf16) k_prepass<__nv_bfloat16><<<grid, kPreThreads, 0, st>>>(bt, GQ);
+  else k_prepass<float><<<grid, kPreThreads, 0, st>>>(bt, GQ);
 }
 
 void launch_logits(const Batch &bt, int maxN, bool bf16, cudaStream_t st) {
@@ -651,17 +595,8 @@ cudaError_t select_configure() {
   return cudaFuncSetAttribute(k_select_gather<float, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn);
 }
 
-cudaError_t euti_configure(int n_qcols, int n_qh, int d, int d_k, int elt) {
+cudaError_t euti_configure(int n_qcols, int n_qh) {
   cudaError_t e = select_configure();
-  if (e != cudaSuccess) return e;
-  // every CTA of the launch reserves the ring; two of them (a streaming one and a Q-reducing one) must
-  // fit on an SM together
-  g_prepass_ring = g_smem_optin > 200 * 1024 ? 92 * 1024 : g_smem_optin / 3;
-  const size_t slot = ((size_t)(d + d_k) * elt + 127) / 128 * 128;
-  if (2 * slot > g_prepass_ring) return cudaErrorInvalidConfiguration;
-  e = cudaFuncSetAttribute(k_prepass<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g_prepass_ring);
-  if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(k_prepass<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g_prepass_ring);
   if (e != cudaSuccess) return e;
   const size_t sm = (size_t)(n_qcols + kRowsPerCta * n_qh) * sizeof(double);
   if (sm > g_smem_optin) return cudaErrorInvalidConfiguration;

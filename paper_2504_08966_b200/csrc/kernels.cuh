@@ -16,7 +16,7 @@ void launch_logits(const Batch &bt, int maxN, bool bf16, cudaStream_t st);
 void launch_scores(const Batch &bt, int maxN, cudaStream_t st);
 // threshold + ordered compaction; gather: also copy the survivor keys and clear the accumulators
 void launch_select_gather(const Batch &bt, int maxN, bool bf16, bool gather, cudaStream_t st);
-cudaError_t euti_configure(int n_qcols, int n_qh, int d, int d_k, int elt);
+cudaError_t euti_configure(int n_qcols, int n_qh);
 cudaError_t select_configure();            // what launch_select_gather needs, once per device
 
 // cluster.cu
