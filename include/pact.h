@@ -117,6 +117,8 @@ typedef struct {
   float *score;         /* [N] EUTI scores; may be NULL                                           */
   uint8_t *keep;        /* [N] 1 = important (survived pruning), 0 = pruned; may be NULL          */
   int32_t *counters;    /* [PACT_N_COUNTERS]                                                      */
+  float *logw_out;      /* [n_total] capacity: log(size_out), the additive attention bias log W of
+                           Eq. 11 for the reduced sequence (0 for text rows); may be NULL           */
 } pact_image;
 
 /* ---- context --------------------------------------------------------------------------- */
@@ -204,8 +206,10 @@ pact_status pact_reincorporate(pact_ctx *ctx, const void *K, int64_t ldK, int N,
 
 /* Merge, Eq. 10 / Algorithm 3 step 4: H_out row (vis_start + c) = mean of the visual rows of H
  * whose label is c (fp32 accumulation in ascending token order), P_out = position id of the
- * centre, size_out = members; text rows are copied around the merged span.
- * Uses img->H, P, H_out, P_out, size_out, counters (N_OUT is written). */
+ * centre, size_out = members, logw_out = log(members) when given (the bias log W that Eq. 11
+ * adds to the attention logits of the reduced sequence; 0 for text rows); text rows are copied
+ * around the merged span.
+ * Uses img->H, P, H_out, P_out, size_out, logw_out, counters (N_OUT is written). */
 pact_status pact_merge(pact_ctx *ctx, const pact_image *img /*host*/, const int32_t *label,
                        const int32_t *center_idx, const int32_t *C_dev, const pact_params *p /*host*/,
                        void *ws, size_t ws_bytes, void *stream);

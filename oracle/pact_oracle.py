@@ -273,6 +273,7 @@ def pact_reduce(H, K_euti, Q_euti, K_clu, P, vis_start, N, n_qh, n_kvh, lam, d_c
         "centers_local": centers_local, "center_idx": center_token, "label": label,
         "dmin_kept": cl["dmin"], "dmin_pruned": dmin_p,
         "H_out": H_out, "P_out": P_out, "size_out": size_out, "n_out": n_out,
+        "logw_out": proportional_attention_bias(size_out),
         "q": int(kept.size), "C": int(C), "r": int((lab_p >= 0).sum()),
         "discarded": int((lab_p < 0).sum()),
         "band_dc": int((np.abs(cl["D"][iu] - dc) <= 1e-6).sum()),

@@ -39,7 +39,8 @@ class ImageDesc(C.Structure):
                 ("P", C.c_void_p), ("n_total", C.c_int32), ("vis_start", C.c_int32), ("N", C.c_int32),
                 ("reserved", C.c_int32), ("H_out", C.c_void_p), ("ldHo", C.c_int64),
                 ("P_out", C.c_void_p), ("size_out", C.c_void_p), ("label", C.c_void_p),
-                ("score", C.c_void_p), ("keep", C.c_void_p), ("counters", C.c_void_p)]
+                ("score", C.c_void_p), ("keep", C.c_void_p), ("counters", C.c_void_p),
+                ("logw_out", C.c_void_p)]
 
 
 _lib = None
@@ -138,13 +139,15 @@ class DeviceImage:
     score: torch.Tensor
     keep: torch.Tensor
     counters: torch.Tensor
+    logw_out: torch.Tensor = None
 
     def desc(self) -> ImageDesc:
         return ImageDesc(_ptr(self.H), self.H.stride(0), _ptr(self.K_euti), self.K_euti.stride(0),
                          _ptr(self.Q_euti), self.Q_euti.stride(0), _ptr(self.K_clu), self.K_clu.stride(0),
                          _ptr(self.P), self.H.shape[0], self.vis_start, self.N, 0,
                          _ptr(self.H_out), self.H_out.stride(0), _ptr(self.P_out), _ptr(self.size_out),
-                         _ptr(self.label), _ptr(self.score), _ptr(self.keep), _ptr(self.counters))
+                         _ptr(self.label), _ptr(self.score), _ptr(self.keep), _ptr(self.counters),
+                         _ptr(self.logw_out))
 
 
 def device_image(img, out_dtype, device="cuda") -> DeviceImage:
@@ -160,7 +163,8 @@ def device_image(img, out_dtype, device="cuda") -> DeviceImage:
                        torch.empty(img.N, dtype=torch.int32, device=device),
                        torch.empty(img.N, dtype=torch.float32, device=device),
                        torch.empty(img.N, dtype=torch.uint8, device=device),
-                       torch.zeros(N_COUNTERS, dtype=torch.int32, device=device))
+                       torch.zeros(N_COUNTERS, dtype=torch.int32, device=device),
+                       torch.empty(n_total, dtype=torch.float32, device=device))
 
 
 class Graph:
@@ -313,14 +317,15 @@ class Context:
 
     def pact_reduce_host(self, host: dict, params: Params, staging: torch.Tensor):
         """host: dict of pinned CPU tensors H, K_euti, Q_euti, K_clu, P, H_out, P_out, size_out,
-        label, counters plus vis_start, N.  Copies in, reduces, copies the valid rows out."""
+        label, counters (and optionally logw_out) plus vis_start, N.  Copies in, reduces, copies the valid rows out."""
         self.ensure_workspace(1, host["N"])
         H = host["H"]
         d = ImageDesc(_ptr(H), H.stride(0), _ptr(host["K_euti"]), host["K_euti"].stride(0),
                       _ptr(host["Q_euti"]), host["Q_euti"].stride(0), _ptr(host["K_clu"]),
                       host["K_clu"].stride(0), _ptr(host["P"]), H.shape[0], host["vis_start"], host["N"], 0,
                       _ptr(host["H_out"]), host["H_out"].stride(0), _ptr(host["P_out"]),
-                      _ptr(host["size_out"]), _ptr(host.get("label")), None, None, _ptr(host["counters"]))
+                      _ptr(host["size_out"]), _ptr(host.get("label")), None, None, _ptr(host["counters"]),
+                      _ptr(host.get("logw_out")))
         w, n = self._ws()
         _check(self.handle, self._L.pact_reduce_host(self.handle, C.byref(d), C.byref(params),
                                                      _ptr(staging), C.c_size_t(staging.numel()), w, n, _stream()))

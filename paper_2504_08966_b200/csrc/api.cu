@@ -190,7 +190,7 @@ void fill_user(ImgDesc &m, const pact_image *g) {
 #endif
   m.H = g->H; m.Ke = g->K_euti; m.Q = g->Q_euti; m.Kc = g->K_clu;
   m.ldH = g->ldH; m.ldKe = g->ldKe; m.ldQ = g->ldQ; m.ldKc = g->ldKc; m.ldHo = g->ldHo;
-  m.P = g->P; m.H_out = g->H_out; m.P_out = g->P_out; m.size_out = g->size_out;
+  m.P = g->P; m.H_out = g->H_out; m.P_out = g->P_out; m.size_out = g->size_out; m.logw_out = g->logw_out;
   m.label_user = g->label; m.counters_user = g->counters; m.score_user = g->score;
   m.keep_user = g->keep;
   m.n_total = g->n_total; m.vis_start = g->vis_start; m.N = g->N;
@@ -574,7 +574,7 @@ size_t pact_host_staging_bytes(const pact_ctx *ctx, int n_total, int N) {
   b += rup((size_t)N * ctx->n_qcols * ctx->elt, kAlign);          // Q
   b += rup((size_t)n_total * 4, kAlign);                          // P
   b += rup((size_t)n_total * ctx->d * oe, kAlign);                // H_out
-  b += 2 * rup((size_t)n_total * 4, kAlign);                      // P_out, size_out
+  b += 3 * rup((size_t)n_total * 4, kAlign);                      // P_out, size_out, logw_out
   b += rup((size_t)N * 4, kAlign);                                // label
   b += rup(PACT_N_COUNTERS * 4, kAlign);                          // counters
   return b;
@@ -603,6 +603,7 @@ pact_status pact_reduce_host(pact_ctx *ctx, const pact_image *img, const pact_pa
   char *dH = take(bH), *dKe = take(bK), *dKc = take(bK), *dQ = take(bQ), *dP = take((size_t)nt * 4);
   char *dHo = take(bHo), *dPo = take((size_t)nt * 4), *dSo = take((size_t)nt * 4), *dL = take((size_t)N * 4);
   char *dC = take(PACT_N_COUNTERS * 4);
+  char *dLw = take((size_t)nt * 4);
   CK(cudaMemcpyAsync(dH, img->H, bH, cudaMemcpyHostToDevice, st));
   CK(cudaMemcpyAsync(dKe, img->K_euti, bK, cudaMemcpyHostToDevice, st));
   const bool alias = img->K_clu == img->K_euti;
@@ -613,6 +614,7 @@ pact_status pact_reduce_host(pact_ctx *ctx, const pact_image *img, const pact_pa
   dv.H = dH; dv.K_euti = dKe; dv.K_clu = alias ? dKe : dKc; dv.Q_euti = dQ; dv.P = (const int32_t *)dP;
   dv.H_out = dHo; dv.P_out = (int32_t *)dPo; dv.size_out = (int32_t *)dSo; dv.label = (int32_t *)dL;
   dv.score = nullptr; dv.keep = nullptr; dv.counters = (int32_t *)dC;
+  dv.logw_out = img->logw_out ? (float *)dLw : nullptr;
   pact_status s = pact_reduce(ctx, &dv, 1, p, 0, ws, ws_bytes, stream);
   if (s != PACT_OK) return s;
   // The number of valid output rows is data dependent: read the counters first, then copy
@@ -624,6 +626,7 @@ pact_status pact_reduce_host(pact_ctx *ctx, const pact_image *img, const pact_pa
   CK(cudaMemcpyAsync(img->H_out, dHo, (size_t)n_out * ctx->d * oe, cudaMemcpyDeviceToHost, st));
   CK(cudaMemcpyAsync(img->P_out, dPo, (size_t)n_out * 4, cudaMemcpyDeviceToHost, st));
   CK(cudaMemcpyAsync(img->size_out, dSo, (size_t)n_out * 4, cudaMemcpyDeviceToHost, st));
+  if (img->logw_out) CK(cudaMemcpyAsync(img->logw_out, dLw, (size_t)n_out * 4, cudaMemcpyDeviceToHost, st));
   if (img->label) CK(cudaMemcpyAsync(img->label, dL, (size_t)N * 4, cudaMemcpyDeviceToHost, st));
   CK(cudaStreamSynchronize(st));
   return PACT_OK;

@@ -22,6 +22,7 @@ struct ImgDesc {
   const int32_t *P;
   void *H_out;
   int32_t *P_out, *size_out, *label_user, *counters_user;
+  float *logw_out;
   float *score_user;
   unsigned char *keep_user;
   int n_total, vis_start, N;

@@ -359,6 +359,7 @@ k_merge(const __grid_constant__ Batch bt) {
     if (t == 0) {
       im.P_out[dst] = im.P[ptok];
       im.size_out[dst] = size;
+      if (im.logw_out) im.logw_out[dst] = logf((float)size);   // Eq. 11: log of the token weight
     }
     u = s_next;
   }

@@ -49,6 +49,7 @@ def gpu_reduce(wl, out_dtype=None, params=None, **over):
             "H_out": im.H_out[:n_out].to(torch.float64).cpu().numpy(),
             "H_out_raw": im.H_out[:n_out].cpu(),
             "P_out": im.P_out[:n_out].cpu().numpy(), "size_out": im.size_out[:n_out].cpu().numpy(),
+            "logw_out": im.logw_out[:n_out].cpu().numpy().astype(np.float64),
         })
     return outs, ctx
 
@@ -101,6 +102,9 @@ def compare_image(o, g, img, out_is_bf16, check_scores=True):
         bad.append("P_out differs")
     if not np.array_equal(g["size_out"], o["size_out"]):
         bad.append("size_out differs")
+    # Eq. 11 bias: fp32 logarithm of an exact integer, two units in the last place
+    if (np.abs(g["logw_out"] - o["logw_out"]) > 2.4e-7 * np.maximum(o["logw_out"], 1.0)).any():
+        bad.append("logw_out differs from log(size_out)")
     ref = o["H_out"]
     if out_is_bf16:
         want = bf16_round(ref)

@@ -300,6 +300,7 @@ def test_reduce_host_matches_device_path():
     host = dict(H=pin(img.H), K_euti=pin(img.K), Q_euti=pin(img.Q), P=pin(img.P), vis_start=img.vis_start, N=img.N,
                 H_out=torch.empty_like(img.H).pin_memory(), P_out=torch.empty(img.n_total, dtype=torch.int32).pin_memory(),
                 size_out=torch.empty(img.n_total, dtype=torch.int32).pin_memory(),
+                logw_out=torch.empty(img.n_total, dtype=torch.float32).pin_memory(),
                 label=torch.empty(img.N, dtype=torch.int32).pin_memory(), counters=torch.zeros(16, dtype=torch.int32).pin_memory())
     host["K_clu"] = host["K_euti"]
     staging = torch.empty(ctx.host_staging_bytes(img.n_total, img.N), dtype=torch.uint8, device="cuda")
@@ -308,6 +309,7 @@ def test_reduce_host_matches_device_path():
     n_out = int(host["counters"][0])
     assert n_out == o["n_out"] and np.array_equal(host["label"].numpy(), o["label"])
     assert np.array_equal(host["P_out"][:n_out].numpy(), o["P_out"])
+    assert np.allclose(host["logw_out"][:n_out].numpy(), o["logw_out"], rtol=2.4e-7, atol=2.4e-7)
     outs, _ = gpu_reduce(wl, torch.bfloat16)
     assert torch.equal(host["H_out"][:n_out].view(torch.int16), outs[0]["H_out_raw"].view(torch.int16))
 
