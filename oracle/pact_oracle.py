@@ -18,6 +18,9 @@ Steps and the passages they follow
 * ``reincorporate``       Eq. 8-9 / Algorithm 3 step 3
 * ``merge``               Eq. 10 / Algorithm 3 step 4 (mean of members; centre's position id)
 * ``proportional_attention_bias``  Eq. 11 (log of the cluster sizes)
+* ``max_key_distance``, ``select_layer``  choice of the reduction layer L (the paragraph after
+  Eq. 11 and the figure it refers to: largest distance between two visual keys of a layer;
+  the earliest layer where it is high enough)
 * ``pact_reduce``         Algorithm 3 end to end
 
 Readings taken where the paper is silent or garbled (each is also listed in the
@@ -31,7 +34,9 @@ d_ii = 0; density ties go to the lower token index; a centre needs distance
 strictly greater than d_c to every earlier centre; argmin ties go to the
 centre with the lowest token index; cluster ids number the centres by
 ascending token index; reincorporation needs distance strictly below
-float32(alpha)*float32(d_c).
+float32(alpha)*float32(d_c); the distance between keys that decides the layer is
+the cosine distance of Eq. 5 on the full key vectors, "sufficiently high" is
+>= a threshold the caller gives, and no layer qualifying is reported as -1.
 
 Pins: every function here is pinned by tests/test_oracle_pins.py against closed
 forms, brute force on tiny inputs, invariants of Appendix B and degenerate
@@ -225,6 +230,19 @@ def merge(Hv: np.ndarray, label: np.ndarray, n_clusters: int, center_token: np.n
 def proportional_attention_bias(sizes: np.ndarray) -> np.ndarray:
     """Eq. 11: the additive logit bias log(w) of a merged token that stands for w tokens."""
     return np.log(sizes.astype(np.float64))
+
+
+def max_key_distance(K: np.ndarray) -> float:
+    """Largest distance (Eq. 5) between two of the visual keys of one layer; 0 for a single key."""
+    return float(cosine_distance(K).max())
+
+
+def select_layer(K_layers, threshold: float) -> int:
+    """The earliest layer whose largest key distance is at least `threshold`; -1 if there is none."""
+    for layer, K in enumerate(K_layers):
+        if max_key_distance(K) >= threshold:
+            return layer
+    return -1
 
 
 # --------------------------------------------------------------------------

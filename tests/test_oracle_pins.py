@@ -315,6 +315,45 @@ def test_proportional_attention_bias_equals_copies():
     assert np.allclose(a, b, atol=1e-14)
 
 
+# ------------------------------------------------------------------ choice of the layer L
+
+def test_max_key_distance_closed_forms():
+    """Known angles in the plane: the largest distance is 1 - cos of the widest angle."""
+    ang = np.deg2rad([0.0, 20.0, 75.0, 130.0])
+    K = np.stack([np.cos(ang), np.sin(ang)], axis=1) * np.array([[1.0], [7.0], [0.25], [3.0]])
+    assert abs(orc.max_key_distance(K) - (1.0 - math.cos(math.radians(130.0)))) < 1e-14
+    assert orc.max_key_distance(np.eye(5)) == 1.0                       # orthogonal keys
+    assert orc.max_key_distance(np.array([[1.0, 2.0], [-2.0, -4.0]])) == 2.0   # opposite keys
+    assert orc.max_key_distance(np.tile([[0.3, -1.0, 2.0]], (6, 1))) == 0.0    # identical keys
+    assert orc.max_key_distance(np.array([[5.0, 1.0]])) == 0.0                 # one key
+
+
+def test_max_key_distance_brute_force_and_scale_invariance():
+    r = _rng(21)
+    K = r.standard_normal((23, 7))
+    best = 0.0
+    for i, j in itertools.combinations(range(23), 2):
+        c = sum(K[i, t] * K[j, t] for t in range(7)) / math.sqrt(sum(x * x for x in K[i]) * sum(x * x for x in K[j]))
+        best = max(best, 1.0 - c)
+    assert abs(orc.max_key_distance(K) - best) < 1e-13
+    assert abs(orc.max_key_distance(K * r.uniform(0.1, 9.0, (23, 1))) - best) < 1e-13
+    assert abs(orc.max_key_distance(K[r.permutation(23)]) - best) < 1e-13
+
+
+def test_select_layer_takes_the_earliest_qualifying_layer():
+    def fan(deg, n=9):
+        a = np.deg2rad(np.linspace(0.0, deg, n))
+        return np.stack([np.cos(a), np.sin(a)], axis=1)
+    layers = [fan(10), fan(25), fan(60), fan(120), fan(40)]
+    spreads = [1.0 - math.cos(math.radians(x)) for x in (10, 25, 60, 120, 40)]
+    assert np.allclose([orc.max_key_distance(K) for K in layers], spreads, atol=1e-14)
+    assert orc.select_layer(layers, 0.4) == 2            # 1 - cos 60 = 0.5 is the first >= 0.4
+    assert orc.select_layer(layers, 0.5 - 1e-12) == 2 and orc.select_layer(layers, 0.5 + 1e-9) == 3
+    assert orc.select_layer(layers, 0.0) == 0
+    assert orc.select_layer(layers, 1.6) == -1
+    assert orc.select_layer(layers[::-1], 0.2) == 0      # order matters: earliest, not largest
+
+
 # ------------------------------------------------------------------ the whole step (Algorithm 3)
 
 @pytest.fixture(scope="module")
