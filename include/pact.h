@@ -204,6 +204,20 @@ pact_status pact_reincorporate(pact_ctx *ctx, const void *K, int64_t ldK, int N,
                                const pact_params *p /*host*/, int32_t *label, int32_t *r_dev,
                                int32_t *counters, void *ws, size_t ws_bytes, void *stream);
 
+/* Choice of the reduction layer L (the paragraph that follows Eq. 11 and the figure it cites): the
+ * earliest layer whose visual keys are spread widely enough.  K_layers is a HOST array of n_layers
+ * DEVICE pointers, each a [N, n_kvh*d_h] key matrix with row stride ldK elements (keys before the
+ * rotary embedding, as in that figure).  For every layer l, max_dist[l] (device, [n_layers]) receives
+ * the largest cosine distance (Eq. 5) between two of its N keys, 0 when N = 1; layer_out (device,
+ * [1], may be NULL) receives the smallest l with max_dist[l] >= threshold, or -1 when no layer
+ * qualifies.  Distances are formed in the arithmetic of pact_dbdpc (fp32 for bf16 keys, fp64 rounded
+ * to fp32 for fp32 keys).  ws must hold pact_workspace_bytes(ctx, min(n_layers, 16), N) bytes.
+ * Asynchronous on `stream`; INVALID_ARG for null or misaligned pointers, n_layers < 1, N < 1, a bad
+ * stride or a NaN threshold, before anything is launched. */
+pact_status pact_key_spread(pact_ctx *ctx, const void *const *K_layers /*host*/, int n_layers, int64_t ldK,
+                            int N, float threshold, float *max_dist, int32_t *layer_out, void *ws,
+                            size_t ws_bytes, void *stream);
+
 /* Merge, Eq. 10 / Algorithm 3 step 4: H_out row (vis_start + c) = mean of the visual rows of H
  * whose label is c (fp32 accumulation in ascending token order), P_out = position id of the
  * centre, size_out = members, logw_out = log(members) when given (the bias log W that Eq. 11

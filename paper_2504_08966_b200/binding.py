@@ -25,7 +25,8 @@ EXPORTS = ["pact_create", "pact_destroy", "pact_workspace_bytes", "pact_status_s
            "pact_last_cuda_error", "pact_importance", "pact_prune", "pact_dbdpc",
            "pact_prune_static", "pact_reincorporate", "pact_merge", "pact_reduce", "pact_reduce_host",
            "pact_host_staging_bytes", "pact_launch_count", "pact_profile_enable", "pact_profile_read",
-           "pact_profile_stage_name", "pact_graph_create", "pact_graph_launch", "pact_graph_destroy"]
+           "pact_profile_stage_name", "pact_graph_create", "pact_graph_launch", "pact_graph_destroy",
+           "pact_key_spread"]
 
 
 class Params(C.Structure):
@@ -68,6 +69,7 @@ def lib():
         L.pact_dbdpc.argtypes = [vp, vp, i64, i32, vp, vp, C.POINTER(Params), vp, vp, vp, vp, vp, vp, sz, vp]
         L.pact_reincorporate.argtypes = [vp, vp, i64, i32, vp, vp, vp, vp, C.POINTER(Params), vp, vp, vp,
                                          vp, sz, vp]
+        L.pact_key_spread.argtypes = [vp, C.POINTER(vp), i32, i64, i32, C.c_float, vp, vp, vp, sz, vp]
         L.pact_merge.argtypes = [vp, C.POINTER(ImageDesc), vp, vp, vp, C.POINTER(Params), vp, sz, vp]
         L.pact_reduce.argtypes = [vp, C.POINTER(ImageDesc), i32, C.POINTER(Params), i32, vp, sz, vp]
         L.pact_reduce_host.argtypes = [vp, C.POINTER(ImageDesc), C.POINTER(Params), vp, sz, vp, sz, vp]
@@ -265,6 +267,16 @@ class Context:
                                                        _ptr(m_dev), _ptr(center_idx), _ptr(C_dev),
                                                        C.byref(params), _ptr(label), _ptr(r_dev),
                                                        _ptr(counters), w, n, _stream()))
+
+    def pact_key_spread(self, K_layers, threshold: float, max_dist, layer_out=None):
+        """K_layers: list of [N, d_k] key matrices (same N and row stride), one per layer."""
+        N, ld = K_layers[0].shape[0], K_layers[0].stride(0)
+        assert all(K.shape[0] == N and K.stride(0) == ld for K in K_layers)
+        self.ensure_workspace(min(len(K_layers), 16), N)
+        arr = (C.c_void_p * len(K_layers))(*[K.data_ptr() for K in K_layers])
+        w, n = self._ws()
+        _check(self.handle, self._L.pact_key_spread(self.handle, arr, len(K_layers), ld, N, float(threshold),
+                                                    _ptr(max_dist), _ptr(layer_out), w, n, _stream()))
 
     def pact_merge(self, im: DeviceImage, label, center_idx, C_dev, params: Params):
         self.ensure_workspace(1, im.N)

@@ -388,6 +388,42 @@ pact_status pact_dbdpc(pact_ctx *ctx, const void *K, int64_t ldK, int N, const i
   return PACT_OK;
 }
 
+pact_status pact_key_spread(pact_ctx *ctx, const void *const *K_layers, int n_layers, int64_t ldK, int N,
+                            float threshold, float *max_dist, int32_t *layer_out, void *ws, size_t ws_bytes,
+                            void *stream) {
+  if (!ctx || !K_layers || !max_dist || n_layers < 1 || N < 1) return PACT_ERR_INVALID_ARG;
+  if (!ld_ok(ctx, ldK, ctx->d_k) || !(threshold == threshold)) return PACT_ERR_INVALID_ARG;
+  for (int l = 0; l < n_layers; ++l)
+    if (!K_layers[l] || !aligned16(K_layers[l])) return PACT_ERR_INVALID_ARG;
+  const int per = n_layers < kMaxBatchPerLaunch ? n_layers : kMaxBatchPerLaunch;
+  pact_status s = check_ws(ctx, ws, ws_bytes, per, N);
+  if (s != PACT_OK) return s;
+  cudaStream_t st = (cudaStream_t)stream;
+  const bool bf = ctx->in == PACT_BF16;
+  const size_t per_img = carve_image(ctx, N, nullptr, nullptr);
+  // the layers go through the tile kernels sixteen at a time, each as one image of a batch
+  for (int base = 0; base < n_layers; base += kMaxBatchPerLaunch) {
+    const int B = n_layers - base < kMaxBatchPerLaunch ? n_layers - base : kMaxBatchPerLaunch;
+    Batch bt;
+    memset(&bt, 0, sizeof(bt));
+    set_dims(ctx, bt, B);
+    for (int b = 0; b < B; ++b) {
+      ImgDesc &m = bt.img[b];
+      carve_image(ctx, N, (char *)ws + (size_t)b * per_img, &m);
+      m.N = N; m.Kc = K_layers[base + b]; m.ldKc = ldK;
+      point_counts_at_workspace(m);
+      CK(cudaMemsetAsync(m.cnt, 0, 32 * sizeof(int32_t), st));
+    }
+    launch_key_rnorm(bt, N, bf, st);
+    if (ctx->umma) CK(launch_spread_umma(bt, N, ctx->ccfg, st));
+    else launch_spread(bt, N, bf, ctx->ccfg, st);
+    launch_spread_finish(bt, max_dist, layer_out, base, threshold, st);
+    ctx->launches += 3;
+    CK(cudaGetLastError());
+  }
+  return PACT_OK;
+}
+
 pact_status pact_reincorporate(pact_ctx *ctx, const void *K, int64_t ldK, int N, const int32_t *pruned_idx,
                                const int32_t *m_dev, const int32_t *center_idx, const int32_t *C_dev,
                                const pact_params *p, int32_t *label, int32_t *r_dev, int32_t *counters,

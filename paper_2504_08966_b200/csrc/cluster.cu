@@ -205,6 +205,77 @@ __global__ void __launch_bounds__(256) k_gram_simt(const __grid_constant__ Batch
   if (band) atomicAdd(&im.cnt[PACT_CNT_BAND_DC], band);
 }
 
+// ---- choice of the reduction layer: largest distance between two keys of a layer ---------------
+// Each image of the batch is one layer's key matrix (Kc, N rows).  Inverse norms first (one warp per
+// key), then the tiles on and above the diagonal with a max-epilogue; the result accumulates in
+// cnt[kCntSpread] as the bit pattern of a non-negative float.
+template <typename T>
+__global__ void __launch_bounds__(256) k_key_rnorm(const __grid_constant__ Batch bt) {
+  using D = typename DistOf<T>::type;
+  using rn_t = typename D::rn_t;
+  const ImgDesc &im = bt.img[blockIdx.y];
+  const int lane = threadIdx.x & 31;
+  const int i = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (i >= im.N) return;
+  const T *row = reinterpret_cast<const T *>(im.Kc) + (size_t)i * im.ldKc;
+  const double ss = row_sumsq<T>(row, bt.d_k, lane);
+  if (lane == 0) rn_tok<D>(im)[i] = (rn_t)(1.0 / sqrt(fmax(ss, 1e-40)));
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) k_spread_simt(const __grid_constant__ Batch bt) {
+  using D = typename DistOf<T>::type;
+  using acc_t = typename D::acc_t;
+  const ImgDesc &im = bt.img[blockIdx.y];
+  const int N = im.N;
+  const int nt = (N + TS - 1) / TS;
+  const int t = threadIdx.x, ty = t >> 4, tx = t & 15;
+  __shared__ __align__(16) float As[KC][TS + 4];
+  __shared__ __align__(16) float Bs[KC][TS + 4];
+  const T *K = reinterpret_cast<const T *>(im.Kc);
+  const auto *rn = rn_tok<D>(im);
+  float mx = 0.f;
+  for (int tile = blockIdx.x; tile < nt * nt; tile += gridDim.x) {
+    const int tm = tile / nt, tn = tile % nt;
+    if (tn < tm) continue;                         // every unordered pair once (uniform)
+    acc_t acc[4][4];
+    tile_dots<T, acc_t>(
+        [&](int r) { const int g = tm * TS + r; return g < N ? K + (size_t)g * im.ldKc : (const T *)nullptr; },
+        [&](int r) { const int g = tn * TS + r; return g < N ? K + (size_t)g * im.ldKc : (const T *)nullptr; },
+        bt.d_k, As, Bs, acc);
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+      const int gi = tm * TS + ty * 4 + a;
+      if (gi >= N) continue;
+      const auto rni = rn[gi];
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        const int gj = tn * TS + tx * 4 + b;
+        if (gj >= N || gj == gi) continue;
+        mx = fmaxf(mx, (float)D::dist(acc[a][b], rni, rn[gj]));
+      }
+    }
+  }
+  const unsigned w = __reduce_max_sync(0xffffffffu, __float_as_uint(mx));   // distances are >= 0
+  if ((t & 31) == 0 && w) atomicMax(reinterpret_cast<unsigned *>(&im.cnt[kCntSpread]), w);
+}
+
+// one warp: max_dist[l] of the layers of this batch, and the earliest layer at or above the threshold
+__global__ void k_spread_finish(const __grid_constant__ Batch bt, float *max_dist, int32_t *layer_out,
+                                int layer_base, float threshold) {
+  const int l = threadIdx.x;
+  float v = -1.f;
+  if (l < bt.B) {
+    v = __int_as_float(bt.img[l].cnt[kCntSpread]);
+    max_dist[layer_base + l] = v;
+  }
+  const unsigned hit = __ballot_sync(0xffffffffu, l < bt.B && v >= threshold);
+  if (l == 0 && layer_out) {
+    if (layer_base == 0) *layer_out = -1;
+    if (hit && *layer_out < 0) *layer_out = layer_base + (__ffs(hit) - 1);
+  }
+}
+
 // ---- centre selection -------------------------------------------------------------------------
 // The sequential loop of Algorithm 2 picks the lexicographically first maximal independent set of
 // the graph {d_ij <= d_c} in density order (ties: lower index first); that set is unique, so any
@@ -616,6 +687,22 @@ void launch_assign(const Batch &bt, int maxN, bool bf16, RowMode mode, const Clu
   const long long nt = (maxN + TS - 1) / TS;
   dim3 grid(tile_grid(nt * nt, cfg.sm_count * 8), bt.B);
   PACT_DISPATCH(bf16, k_assign_simt, <<<grid, 256, 0, st>>>(bt, (int)mode));
+}
+
+void launch_key_rnorm(const Batch &bt, int maxN, bool bf16, cudaStream_t st) {
+  dim3 grid((maxN + 7) / 8, bt.B);
+  PACT_DISPATCH(bf16, k_key_rnorm, <<<grid, 256, 0, st>>>(bt));
+}
+
+void launch_spread(const Batch &bt, int maxN, bool bf16, const ClusterCfg &cfg, cudaStream_t st) {
+  const long long nt = (maxN + TS - 1) / TS;
+  dim3 grid(tile_grid(nt * (nt + 1) / 2, cfg.sm_count * 8), bt.B);
+  PACT_DISPATCH(bf16, k_spread_simt, <<<grid, 256, 0, st>>>(bt));
+}
+
+void launch_spread_finish(const Batch &bt, float *max_dist, int32_t *layer_out, int layer_base, float threshold,
+                          cudaStream_t st) {
+  k_spread_finish<<<1, 32, 0, st>>>(bt, max_dist, layer_out, layer_base, threshold);
 }
 
 void launch_label(const Batch &bt, int maxN, bool bf16, RowMode mode, cudaStream_t st) {

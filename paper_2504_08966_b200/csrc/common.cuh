@@ -12,6 +12,7 @@ constexpr int kMaxBatchPerLaunch = 16;   // images described by one kernel param
 constexpr int kRowsPerCta = 32;          // visual tokens handled by one CTA of the EUTI kernels
 constexpr uint32_t kRhoShift = 30;       // density terms are summed as integers scaled by 2^30
 constexpr unsigned long long kBestInit = 0xFFFFFFFFFFFFFFFFull;
+constexpr int kCntSpread = 24;           // slot of cnt[]: largest key distance of a layer, as float bits
 constexpr int kSpinLimit = 1 << 20;      // passes a centre-selection warp makes before it gives up
 
 // Per-image device pointers: the caller's buffers and the slices of the workspace.

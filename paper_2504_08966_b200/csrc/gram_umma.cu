@@ -1,7 +1,9 @@
 // tcgen05 tile kernels for bf16 keys (sm_100a): the all-pairs distance pass of DBDPC (Eq. 5) with
-// the density (Eq. 6) and the d <= d_c adjacency fused into the epilogue, and the rows x centres
-// nearest-centre pass (Algorithm 2 assignment, Eq. 8).  Nothing of the distance matrix reaches
-// memory: accumulators live in tensor memory and are consumed from there.
+// the density (Eq. 6) and the d <= d_c adjacency fused into the epilogue, the rows x centres
+// nearest-centre pass (Algorithm 2 assignment, Eq. 8), and the largest distance between two keys of a
+// layer (the quantity that decides the reduction layer L) as a max-epilogue over the tiles on and above
+// the diagonal.  Nothing of the distance matrix reaches memory: accumulators live in tensor memory
+// and are consumed from there.
 //
 // One persistent CTA per SM, 320 threads:
 //   warp 0      TMA producer: 128-byte-swizzled K-slabs of the two operands into a shared-memory ring
@@ -94,7 +96,13 @@ struct Shared {
   __align__(16) float rn_col[EPI_WARPS][HALF];   // inverse norms of this warp's columns
 };
 
-enum { MODE_GRAM = 0, MODE_ASSIGN = 1 };
+enum { MODE_GRAM = 0, MODE_ASSIGN = 1, MODE_SPREAD = 2 };
+
+// The largest-distance pass needs every unordered pair once: tiles that lie wholly below the diagonal
+// are left out (by the producer, the MMA issuer and the epilogue alike).
+template <int MODE> __device__ __forceinline__ bool tile_wanted(int tmi, int tni) {
+  return MODE != MODE_SPREAD || (tni + 1) * BN > tmi * BM;
+}
 
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
@@ -159,6 +167,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
                                                            const __grid_constant__ TmapSet tm, int kept_rows) {
   const ImgDesc &im = bt.img[blockIdx.y];
   TL_SCOPE(im, MODE == MODE_GRAM ? 4 : 6);
+  (void)kept_rows;
   extern __shared__ uint8_t smem_raw[];
   __shared__ Shared sh;
   uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -166,6 +175,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
 
   int nrows, ncols;
   if (MODE == MODE_GRAM) { nrows = *im.q_ptr; ncols = nrows; }
+  else if (MODE == MODE_SPREAD) { nrows = im.N; ncols = im.N; }
   else { nrows = kept_rows ? *im.q_ptr : im.N; ncols = *im.C_ptr; }
   const int ntm = (nrows + BM - 1) / BM, ntn = (ncols + BN - 1) / BN;
   const int ntiles = ntm * ntn;
@@ -192,6 +202,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < ntiles; tile += gridDim.x) {
         const int tmi = tile / ntn, tni = tile % ntn;
+        if (!tile_wanted<MODE>(tmi, tni)) continue;
         for (int ks = 0; ks < nslab; ++ks, ++it) {
           const int s = it % STAGES;
           if (!mbar_wait(&sh.empty[s], ((it / STAGES) & 1) ^ 1)) { ok = false; break; }
@@ -215,7 +226,8 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
     if (lane == 0) {
       uint32_t it = 0, tcount = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < ntiles; tile += gridDim.x, ++tcount) {
+      for (int tile = blockIdx.x; ok && tile < ntiles; tile += gridDim.x) {
+        if (!tile_wanted<MODE>(tile / ntn, tile % ntn)) continue;
         const uint32_t a = tcount & 1;
         if (!mbar_wait(&sh.acc_empty[a], ((tcount >> 1) & 1) ^ 1)) { ok = false; break; }
         tc_fence_after();
@@ -231,6 +243,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
           umma_commit(&sh.empty[s]);               // frees the slab once these MMAs have read it
         }
         if (ok) umma_commit(&sh.acc_full[a]);      // accumulator complete
+        ++tcount;
       }
       if (!ok) atomicExch(&sh.abort, 1);
     }
@@ -243,12 +256,14 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
     uint32_t tcount = 0;
     int band = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; ok && tile < ntiles; tile += gridDim.x, ++tcount) {
+    float mx = 0.f;                                 // largest distance seen by this lane (MODE_SPREAD)
+    for (int tile = blockIdx.x; ok && tile < ntiles; tile += gridDim.x) {
       const int tmi = tile / ntn, tni = tile % ntn;
+      if (!tile_wanted<MODE>(tmi, tni)) continue;
       const uint32_t a = tcount & 1;
       const int cbase = tni * BN + half * HALF;     // first column of this warp
       // inverse norms of this warp's columns and of this lane's row (in flight while the MMAs run)
-      const float *rn_src = MODE == MODE_GRAM ? im.rnk : im.rnc;
+      const float *rn_src = MODE == MODE_GRAM ? im.rnk : (MODE == MODE_SPREAD ? im.rn : im.rnc);
       float4 r4;
       {
         const int gj = cbase + lane * 4;
@@ -259,7 +274,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
       }
       const int row = tmi * BM + qd * 32 + lane;
       const bool row_ok = row < nrows;
-      const bool kept_space = MODE == MODE_GRAM || kept_rows;
+      const bool kept_space = MODE == MODE_GRAM || (MODE == MODE_ASSIGN && kept_rows);
       const float rni = row_ok ? (kept_space ? im.rnk[row] : im.rn[row]) : 0.f;
       __syncwarp();
       reinterpret_cast<float4 *>(rn_col)[lane] = r4;
@@ -289,6 +304,21 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
             if (row < c0) band += bnd;              // each unordered pair once; the chunk lies wholly on one side
           }
           if (row_ok) im.adj[(size_t)row * im.Wp + (c0 >> 5)] = bits;
+        } else if (MODE == MODE_SPREAD) {
+          // rows and columns past the end hold zero dot products, i.e. distance 1: leave them out
+          const int lim = row_ok ? min(32, ncols - c0) : 0;
+          const int self = row - c0;                 // the pair (i, i) is not a pair
+#pragma unroll
+          for (int k4 = 0; k4 < 32; k4 += 4) {
+            const float4 rn4 = *reinterpret_cast<const float4 *>(rn_col + ch * 32 + k4);
+            const float rnj[4] = {rn4.x, rn4.y, rn4.z, rn4.w};
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+              const int k = k4 + kk;
+              const float dd = DistF::dist(__uint_as_float(v[k]), rni, rnj[kk]);
+              if (k < lim && k != self) mx = fmaxf(mx, dd);
+            }
+          }
         } else {
           const int lim = min(32, ncols - c0);
 #pragma unroll
@@ -308,9 +338,10 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh.acc_empty[a]);
+      ++tcount;
       if (row_ok) {
         if (MODE == MODE_GRAM) atomicAdd(&im.rho_fix[row], rowsum);
-        else if (bd <= 2.0f) {
+        else if (MODE == MODE_ASSIGN && bd <= 2.0f) {
           const unsigned long long pk = ((unsigned long long)__float_as_uint(bd) << 32) | (unsigned)bi;
           atomicMin(&im.best[kept_rows ? im.kept_idx[row] : row], pk);
         }
@@ -318,6 +349,11 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
     }
     if (!ok) atomicExch(&sh.abort, 1);
     if (MODE == MODE_GRAM && band) atomicAdd(&im.cnt[PACT_CNT_BAND_DC], band);
+    if (MODE == MODE_SPREAD) {
+      // distances are clamped to [0, 2]: their bit patterns order like unsigned integers
+      const unsigned w = __reduce_max_sync(0xffffffffu, __float_as_uint(mx));
+      if (lane == 0 && w) atomicMax(reinterpret_cast<unsigned *>(&im.cnt[kCntSpread]), w);
+    }
   }
 
   tc_fence_before();
@@ -359,6 +395,8 @@ cudaError_t umma_configure() {
   g_encode = reinterpret_cast<EncodeTiledFn>(fn);
   e = cudaFuncSetAttribute(k_tiles_umma<MODE_GRAM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kUmmaSmem);
   if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(k_tiles_umma<MODE_SPREAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kUmmaSmem);
+  if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(k_tiles_umma<MODE_ASSIGN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kUmmaSmem);
 }
 
@@ -395,6 +433,19 @@ cudaError_t launch_assign_umma(const Batch &bt, int maxN, bool kept_rows, const 
   }
   dim3 grid(umma_grid_x(maxN, maxN, bt.B, cfg.sm_count), bt.B);
   k_tiles_umma<MODE_ASSIGN><<<grid, THREADS, kUmmaSmem, st>>>(bt, tm, kept_rows ? 1 : 0);
+  return cudaGetLastError();
+}
+
+// every layer of the batch is one "image": rows and columns are all N keys of K_clu
+cudaError_t launch_spread_umma(const Batch &bt, int maxN, const ClusterCfg &cfg, cudaStream_t st) {
+  TmapSet tm;
+  for (int b = 0; b < bt.B; ++b) {
+    const ImgDesc &im = bt.img[b];
+    if (!encode_rows(&tm.a[b], im.Kc, im.N, im.ldKc, bt.d_k)) return cudaErrorInvalidValue;
+    tm.b[b] = tm.a[b];
+  }
+  dim3 grid(umma_grid_x(maxN, maxN, bt.B, cfg.sm_count), bt.B);
+  k_tiles_umma<MODE_SPREAD><<<grid, THREADS, kUmmaSmem, st>>>(bt, tm, 0);
   return cudaGetLastError();
 }
 

@@ -34,12 +34,18 @@ void launch_gram(const Batch &bt, int maxN, bool bf16, const ClusterCfg &cfg, cu
 cudaError_t launch_centers(const Batch &bt, int maxQ, bool bf16, const ClusterCfg &cfg, cudaStream_t st);
 void launch_assign(const Batch &bt, int maxN, bool bf16, RowMode mode, const ClusterCfg &cfg, cudaStream_t st);
 void launch_label(const Batch &bt, int maxN, bool bf16, RowMode mode, cudaStream_t st);
+// layer choice: inverse norms of all keys of every layer, largest pair distance (any dtype), result
+void launch_key_rnorm(const Batch &bt, int maxN, bool bf16, cudaStream_t st);
+void launch_spread(const Batch &bt, int maxN, bool bf16, const ClusterCfg &cfg, cudaStream_t st);
+void launch_spread_finish(const Batch &bt, float *max_dist, int32_t *layer_out, int layer_base, float threshold,
+                          cudaStream_t st);
 
 // gram_umma.cu: tcgen05 versions of the two tile passes for bf16 keys whose width is a multiple of 64
 cudaError_t umma_configure();
 bool umma_supported(int d_k);
 cudaError_t launch_gram_umma(const Batch &bt, int maxN, const ClusterCfg &cfg, cudaStream_t st);
 cudaError_t launch_assign_umma(const Batch &bt, int maxN, bool kept_rows, const ClusterCfg &cfg, cudaStream_t st);
+cudaError_t launch_spread_umma(const Batch &bt, int maxN, const ClusterCfg &cfg, cudaStream_t st);
 
 // merge.cu
 // member lists from label[] (from_best: labels are first formed from the nearest-centre pass, all tokens);

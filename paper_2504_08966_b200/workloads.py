@@ -240,6 +240,28 @@ def stress(seed: int = 4, B: int = 4, N: int = 16384, T: int = 64, n_blobs: int 
     return Workload("stress", imgs, d, n_h, n_h, d_h, dtype, lam, d_c)
 
 
+def layer_keys(seed: int = 5, n_layers: int = 10, N: int = 7290, n_h: int = 4, d_h: int = 128,
+               dtype=torch.bfloat16, mix=None) -> List[torch.Tensor]:
+    """Keys of the visual tokens at the first `n_layers` decoder layers, for the choice of the
+    reduction layer: K_l[i] = gain_i * (shared_l + mix[l] * token_i,l) with a unit shared direction per
+    layer and unit-scale token-specific noise.  With a small mix the keys of a layer are nearly
+    parallel, as the first layers of the paper's model are described; the default mix grows with
+    depth but not monotonically, so that "earliest layer above a threshold" and "layer with the
+    widest keys" differ."""
+    rng = np.random.default_rng(seed)
+    d_k = n_h * d_h
+    if mix is None:
+        base = [0.02, 0.05, 0.04, 0.15, 0.4, 0.3, 0.9, 0.7, 1.5, 1.2]
+        mix = [base[l % len(base)] for l in range(n_layers)]
+    out = []
+    for l in range(n_layers):
+        shared = _unit_rows(rng.standard_normal((1, d_k)))
+        tok = rng.standard_normal((N, d_k)) / np.sqrt(d_k)
+        gain = rng.lognormal(0.0, 0.25, (N, 1))
+        out.append(torch.from_numpy(gain * (shared + mix[l] * tok)).to(dtype).contiguous())
+    return out
+
+
 BUILDERS = {"tiny": tiny, "single_image": single_image, "batched": batched, "video": video,
             "stress": stress}
 
