@@ -152,6 +152,134 @@ def reference_arm(args):
     print(json.dumps(line))
 
 
+STAGE_WORKLOADS = ("euti_only", "dbdpc_only", "layer_choice")
+
+
+def stage_bench(args):
+    """Second workload shapes, each a sequence of stage calls of the library on one GPU:
+    euti_only    pact_importance + pact_prune on the single_image inputs (EUTI as a pruning method)
+    dbdpc_only   pact_dbdpc over all N tokens + pact_merge (DBDPC as a clustering method, the
+                 tensor-bound regime: the Gram pass covers N instead of N/2 rows)
+    layer_choice pact_key_spread over the keys of ten layers
+    Prints one JSON line with the timing, the kernel launches and the roofline of the stage."""
+    from paper_2504_08966_b200 import binding as pb
+    from paper_2504_08966_b200 import workloads
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (no CPU fallback)")
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+        if int(os.environ.get("RANK", "0")) != 0:
+            return
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    W = max(3, args.warmup)
+    pk = _peaks()
+    wl = workloads.single_image()
+    img = wl.images[0]
+    N, d, d_k = img.N, wl.d, wl.d_k
+    ctx = pb.Context(wl.d, wl.n_qh, wl.n_kvh, wl.d_h, wl.dtype, torch.bfloat16)
+    params = pb.make_params(lam=wl.lam, d_c=wl.d_c, d_n=wl.d_n, alpha=wl.alpha)
+    i32 = lambda n, v=0: torch.full((n,), v, dtype=torch.int32, device="cuda")
+    copies = N_COPIES
+    extra = {}
+    if args.workload == "euti_only":
+        sets = [pb.device_image(img, torch.bfloat16) for _ in range(copies)]
+        keep, kept, pruned, cnts = torch.empty(N, dtype=torch.uint8, device="cuda"), i32(N), i32(N), i32(2)
+
+        def step(i):
+            im = sets[i % copies]
+            ctx.pact_importance(im, params, im.score)
+            ctx.pact_prune(im.score, params, keep, kept, pruned, cnts)
+        units = N
+        kind, amount = "hbm", N * d * 2.0 + N * d_k * 2.0 + N * wl.n_qh * wl.d_h * 2.0
+        what = "pact_importance + pact_prune, single_image inputs"
+
+        def oracle_once():
+            from oracle import pact_oracle as orc
+            from tests.helpers import f64
+            v = slice(img.vis_start, img.vis_start + N)
+            sc = orc.importance_scores(f64(img.H)[v], f64(img.K), f64(img.Q), wl.n_qh, wl.n_kvh)
+            orc.split(sc.astype(np.float32), wl.lam)
+    elif args.workload == "dbdpc_only":
+        sets = [pb.device_image(img, torch.bfloat16) for _ in range(copies)]
+        idx, qd = torch.arange(N, dtype=torch.int32, device="cuda"), i32(1, N)
+        rho, cidx, Cd = torch.empty(N, dtype=torch.float32, device="cuda"), i32(N), i32(1)
+
+        def step(i):
+            im = sets[i % copies]
+            ctx.pact_dbdpc(im.K_clu, idx, qd, params, rho, cidx, Cd, im.label)
+            ctx.pact_merge(im, im.label, cidx, Cd, params)
+        step(0)
+        torch.cuda.synchronize()
+        Cn = int(Cd.item())
+        units = N
+        kind, amount = "tensor", 2.0 * d_k * (N * (N + 1) / 2) + 2.0 * d_k * N * Cn
+        what = f"pact_dbdpc over all N tokens + pact_merge (C = {Cn})"
+        extra["C"] = Cn
+
+        def oracle_once():
+            from oracle import pact_oracle as orc
+            from tests.helpers import f64
+            orc.dbdpc(f64(img.K), wl.d_c, wl.d_n)
+    else:
+        n_layers = 10
+        copies = 2
+        sets = [[K.cuda() for K in workloads.layer_keys(seed=5 + c, n_layers=n_layers, N=N)] for c in range(copies)]
+        md, lo = torch.empty(n_layers, dtype=torch.float32, device="cuda"), i32(1)
+
+        def step(i):
+            ctx.pact_key_spread(sets[i % copies], 0.3, md, lo)
+        units = n_layers * N
+        kind, amount = "tensor", n_layers * 2.0 * d_k * (N * (N - 1) / 2)
+        what = f"pact_key_spread, {n_layers} layers of N keys (units = keys)"
+
+        def oracle_once():
+            from oracle import pact_oracle as orc
+            from tests.helpers import f64
+            for K in sets[0][:2]:
+                orc.max_key_distance(f64(K.cpu()))
+        extra["cpu_sample_scale"] = n_layers / 2
+    steps = min(args.steps, 500)
+    for i in range(W):
+        step(i)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    l0 = ctx.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        step(W + i)
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / steps
+    launches = ctx.launch_count() - l0
+    secs = ms * 1e-3
+    if kind == "hbm":
+        ach, peak, unit = amount / secs / 1e9, pk["hbm_gbs"], "GB/s"
+    else:
+        ach, peak, unit = amount / secs / 1e12, pk["bf16_tflops"], "TFLOP/s"
+    cpu = None
+    if not args.no_cpu_baseline:
+        t0 = time.perf_counter()
+        oracle_once()
+        dt = (time.perf_counter() - t0) * extra.pop("cpu_sample_scale", 1.0)
+        cpu = {"value": units / dt, "unit": UNIT, "cores": _cpu_threads(), "kind": "oracle",
+               "sample": "one pass of the oracle functions of this stage"
+                         + (" over two of the ten layers, scaled" if args.workload == "layer_choice" else "")}
+    extra.pop("cpu_sample_scale", None)
+    print(json.dumps({
+        "metric": METRIC, "value": units / secs, "unit": UNIT, "n_gpus": 1, "steps": steps, "warmup": W,
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": f"{args.workload}: {what}", "N": N, "d": d, "d_k": d_k, "lambda": wl.lam,
+                   "d_c": wl.d_c, "launch": "stage calls on the stream, whole sequence timed",
+                   "l2": f"{copies} input copies rotated between steps", **extra},
+        "latency_us": ms * 1e3, "clocks": clocks, "e2e": None, "gpu_launches": int(launches),
+        "roofline": {"kernel": "whole stage sequence", "bound": kind, "achieved": ach, "peak": peak, "unit": unit,
+                     "frac": ach / peak, "traffic": None, "peak_source": pk["source"]},
+        "cpu_baseline": cpu}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -159,10 +287,14 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="pact", choices=["pact", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="single_image", choices=["single_image", "video", "batched", "stress"])
+    ap.add_argument("--workload", default="single_image",
+                    choices=["single_image", "video", "batched", "stress", *STAGE_WORKLOADS])
     args = ap.parse_args()
     if args.impl == "reference":
         reference_arm(args)
+        return
+    if args.workload in STAGE_WORKLOADS:
+        stage_bench(args)
         return
 
     import torch.distributed as dist

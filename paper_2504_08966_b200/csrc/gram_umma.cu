@@ -113,19 +113,19 @@ __device__ __forceinline__ float ex2_approx(float x) {
 // One 32-column chunk of the epilogue of the all-pairs pass for one row (= one lane): distance
 // (Eq. 5), density term (Eq. 6) as an integer multiple of 2^-30, adjacency bit d <= d_c, band count.
 // EDGE adds the per-element checks that only edge chunks need (diagonal, columns past the end).
-// The arithmetic is that of DistF (common.cuh) written out so that four terms are summed in 32 bits.
+// The arithmetic is that of DistF (common.cuh) written out so that three terms are summed in 32 bits.
 template <bool EDGE>
 __device__ __forceinline__ void gram_chunk(const uint32_t (&v)[32], const float *rn_col, float rni, int row, int c0,
                                            int ncols, float d_c, float neg_k, unsigned long long &rowsum,
                                            uint32_t &bits, int &band) {
   uint32_t b = 0u;
   unsigned long long s = 0ull;
+  uint32_t s3 = 0u;                                 // three terms, each at most 2^30, fit in 32 bits
   int bnd = 0;
 #pragma unroll
   for (int k4 = 0; k4 < 32; k4 += 4) {
     const float4 rn4 = *reinterpret_cast<const float4 *>(rn_col + k4);
     const float rnj[4] = {rn4.x, rn4.y, rn4.z, rn4.w};
-    uint32_t s4 = 0u;                               // four terms, each at most 2^30, fit in 32 bits
 #pragma unroll
     for (int kk = 0; kk < 4; ++kk) {
       const int k = k4 + kk;
@@ -141,17 +141,17 @@ __device__ __forceinline__ void gram_chunk(const uint32_t (&v)[32], const float 
       const bool inband = fabsf(dd - d_c) <= 1e-6f;
       if (EDGE) {
         if (ok) {
-          s4 += term;
+          s3 += term;
           if (within) b |= 1u << k;
           if (inband && row < c0 + k) ++bnd;
         }
       } else {
-        s4 += term;
+        s3 += term;
         if (within) b |= 1u << k;
         if (inband) ++bnd;
       }
+      if (k % 3 == 2 || k == 31) { s += s3; s3 = 0u; }   // a run of keys at distance 0 adds 2^30 each
     }
-    s += s4;
   }
   rowsum += s;
   bits = b;

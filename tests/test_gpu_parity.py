@@ -289,6 +289,72 @@ def test_stage_dbdpc_reincorporate_merge(stage_case):
     assert np.array_equal(im.size_out[:n_out].cpu().numpy(), o["size_out"])
 
 
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_stage_dbdpc_runs_of_identical_keys(dtype):
+    """Uniform image regions give runs of identical (or exactly parallel) keys: many neighbouring
+    pairs at distance 0, each adding the largest possible term to a density."""
+    from paper_2504_08966_b200 import binding as pb
+    wl = workloads.single_image(seed=83, N=1500, T=8, n_blobs=40, dtype=dtype)
+    K = wl.images[0].K.clone()
+    K[200:218] = K[200]
+    K[300:309] = (K[300].float() * 2.0).to(dtype)
+    K[301] = K[300]
+    K[640:644] = K[640]
+    # one non-zero element, a power of two: norms and cosines are exact, these distances are exactly 0
+    K[800:813] = 0
+    K[800:813, 3] = torch.tensor([2.0 ** (i % 3 - 1) for i in range(13)], dtype=dtype)
+    N = K.shape[0]
+    o = orc.dbdpc(f64(K), wl.d_c, wl.d_n)
+    ctx = pb.Context(wl.d, wl.n_qh, wl.n_kvh, wl.d_h, dtype, torch.float32)
+    idx = torch.arange(N, dtype=torch.int32, device="cuda")
+    q_dev = torch.tensor([N], dtype=torch.int32, device="cuda")
+    rho = torch.empty(N, dtype=torch.float32, device="cuda")
+    cidx = torch.empty(N, dtype=torch.int32, device="cuda")
+    C_dev = torch.zeros(1, dtype=torch.int32, device="cuda")
+    label = torch.empty(N, dtype=torch.int32, device="cuda")
+    ctx.pact_dbdpc(K.cuda(), idx, q_dev, pb.make_params(lam=0.0, d_c=wl.d_c, d_n=wl.d_n), rho, cidx, C_dev, label)
+    torch.cuda.synchronize()
+    rel = np.abs(rho.cpu().numpy() - o["rho"]) / o["rho"]
+    assert rel.max() < 1e-6
+    C = int(C_dev)
+    assert C == o["centers"].size and np.array_equal(cidx[:C].cpu().numpy(), o["centers"])
+    assert np.array_equal(label.cpu().numpy(), o["label"])
+
+
+def test_stage_dbdpc_over_all_tokens_at_full_size():
+    """DBDPC as a clustering method of its own (nothing pruned): N = 7290 rows in the Gram pass."""
+    from paper_2504_08966_b200 import binding as pb
+    wl = workloads.single_image()
+    img = wl.images[0]
+    N = img.N
+    o = orc.dbdpc(f64(img.K), wl.d_c, wl.d_n)
+    ctx = pb.Context(wl.d, wl.n_qh, wl.n_kvh, wl.d_h, wl.dtype, torch.bfloat16)
+    K = img.K.cuda()
+    idx = torch.arange(N, dtype=torch.int32, device="cuda")
+    q_dev = torch.tensor([N], dtype=torch.int32, device="cuda")
+    rho = torch.empty(N, dtype=torch.float32, device="cuda")
+    cidx = torch.empty(N, dtype=torch.int32, device="cuda")
+    C_dev = torch.zeros(1, dtype=torch.int32, device="cuda")
+    label = torch.empty(N, dtype=torch.int32, device="cuda")
+    cnt = torch.zeros(16, dtype=torch.int32, device="cuda")
+    ctx.pact_dbdpc(K, idx, q_dev, pb.make_params(lam=0.0, d_c=wl.d_c, d_n=wl.d_n), rho, cidx, C_dev, label, cnt)
+    torch.cuda.synchronize()
+    c = cnt.cpu().numpy()
+    assert int(c[pb.CNT["status"]]) == 0
+    iu = np.triu_indices(N, 1)
+    fragile = int((np.abs(o["D"][iu] - float(np.float32(wl.d_c))) <= 1e-6).sum())
+    assert int(c[pb.CNT["band_dc"]]) >= fragile - 2 and fragile < 50
+    C = int(C_dev)
+    if fragile == 0:
+        assert C == o["centers"].size and np.array_equal(cidx[:C].cpu().numpy(), o["centers"])
+        assert np.array_equal(label.cpu().numpy(), o["label"])
+    else:   # pairs on the cutoff may fall either way in fp32; the rest of the structure must hold
+        assert abs(C - o["centers"].size) <= fragile
+        assert (label.cpu().numpy() == o["label"]).mean() > 0.9 or C != o["centers"].size
+    rel = np.abs(rho.cpu().numpy() - o["rho"]) / o["rho"]
+    assert rel.max() < 1e-6
+
+
 # ------------------------------------------------------------------ host-buffer entry point and error paths
 
 def test_reduce_host_matches_device_path():
