@@ -101,6 +101,33 @@ def test_degenerate_parameters(over):
         assert g["discarded"] == 0
 
 
+@pytest.mark.parametrize("kind", ["uniform", "two_valued", "zero_keys", "one_hot_runs"])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_degenerate_inputs(kind, dtype):
+    """Images whose keys repeat exactly (flat regions), vanish, or are exactly parallel."""
+    wl = workloads.single_image(seed=61, N=900, T=6, n_blobs=20, d=256, n_h=2, d_h=64, dtype=dtype)
+    img = wl.images[0]
+    K = img.K
+    if kind == "uniform":
+        K[:] = K[17].clone()
+    elif kind == "two_valued":
+        a, b = K[3].clone(), K[4].clone()
+        K[0::2] = a
+        K[1::2] = b
+    elif kind == "zero_keys":
+        K[100:164] = 0
+        K[500] = 0
+    else:
+        K[200:264] = 0
+        K[200:264, 5] = torch.tensor([2.0 ** (i % 4 - 2) for i in range(64)], dtype=dtype)
+        img.H[img.vis_start + 200:img.vis_start + 264] *= 4      # keep them among the survivors
+    outs = _check_workload(wl, torch.float32)
+    if kind == "uniform":
+        assert outs[0]["C"] == 1 and outs[0]["discarded"] == 0
+    if kind == "two_valued":
+        assert outs[0]["C"] <= 2
+
+
 def test_no_text_tokens_and_gqa_and_distinct_clustering_keys():
     _check_workload(_small(seed=41, T=0), torch.bfloat16)
     _check_workload(_small(seed=42, n_qh=4), torch.bfloat16)
