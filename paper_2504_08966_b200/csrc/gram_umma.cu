@@ -404,7 +404,7 @@ bool umma_supported(int d_k) { return g_encode != nullptr && d_k % BK == 0; }
 
 static int umma_grid_x(int max_rows, int max_cols, int B, int sms) {
   const long long tiles = (long long)((max_rows + BM - 1) / BM) * ((max_cols + BN - 1) / BN);
-  long long x = (sms + B - 1) / B;
+  long long x = sms / B;                            // one CTA per SM: all CTAs of the batch run at once
   if (x < 1) x = 1;
   if (x > tiles) x = tiles;
   return (int)(x < 1 ? 1 : x);
