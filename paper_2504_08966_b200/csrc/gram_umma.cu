@@ -10,8 +10,10 @@
 //   warp 1      allocates tensor memory, issues tcgen05.mma (128 x BN x 16, bf16 -> fp32)
 //   warps 2-9   epilogue: tcgen05.ld of their 32-lane quadrant (two warps per quadrant, half of the
 //               columns each), distance arithmetic of common.cuh
-// Two accumulators (2 x BN columns of tensor memory) let the epilogue of tile t overlap the MMAs of
-// tile t+1.  Every mbarrier wait is bounded; when one runs out the CTA raises the image's status
+// Several accumulators (512 / BN of them share the tensor memory) let the epilogue of tile t overlap
+// the MMAs of the next tiles.  The all-pairs pass computes every unordered pair of survivors once: a
+// 128 x 128 block above the diagonal serves its rows (density sums, adjacency words) and, through
+// warp-wide sums and ballots, its columns as well; blocks on the diagonal serve their rows only.  Every mbarrier wait is bounded; when one runs out the CTA raises the image's status
 // word, drains what it armed, frees its tensor memory and returns.
 #include <cuda.h>
 
@@ -23,13 +25,27 @@ namespace pact {
 namespace {
 
 constexpr int BM = 128;           // rows per tile (UMMA M)
-constexpr int BN = 256;           // columns per tile (UMMA N)
 constexpr int BK = 64;            // bf16 elements per K-slab = one 128-byte swizzle row
-constexpr int STAGES = 4;
 constexpr int A_BYTES = BM * BK * 2;
-constexpr int B_BYTES = BN * BK * 2;
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int TMEM_COLS = 2 * BN; // 512: all of an SM's tensor memory
+constexpr int TMEM_COLS = 512;    // all of an SM's tensor memory
+constexpr int MAX_STAGES = 6;
+constexpr int MAX_ACC = 4;
+
+// Per tile width BN (UMMA N): 256 columns for the rows x centres and the largest-distance passes,
+// 128 for the all-pairs pass, whose tiles are the 128 x 128 blocks on and above the diagonal.
+template <int BN> struct TileCfg {
+  static constexpr int B_BYTES = BN * BK * 2;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int STAGES = BN == 256 ? 4 : 5;
+  static constexpr int NACC = TMEM_COLS / BN;      // accumulators in tensor memory
+  static constexpr int HALF = BN / 2;              // columns per epilogue warp
+  // BN = 128 (all-pairs pass): one 32 x 32 exchange buffer per epilogue warp behind the ring
+  static constexpr size_t RING = 1024 + (size_t)STAGES * STAGE_BYTES;
+  static constexpr size_t SMEM = RING + (BN == 128 ? (size_t)8 * 32 * 36 * 4 : 0);
+  // kind::f16 instruction descriptor: fp32 accumulate, bf16 x bf16, both operands K-major.
+  static constexpr uint32_t IDESC =
+      (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+};
 
 struct TmapSet {
   CUtensorMap a[kMaxBatchPerLaunch];
@@ -82,26 +98,43 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
   return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
          ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
 }
-// kind::f16 instruction descriptor: fp32 accumulate, bf16 x bf16, both operands K-major.
-constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-
 constexpr int EPI_WARPS = 8;      // two per tensor-memory lane quadrant; each takes half of the columns
 constexpr int THREADS = 64 + EPI_WARPS * 32;
-constexpr int HALF = BN / 2;      // columns per epilogue warp
 
 struct Shared {
-  uint64_t full[STAGES], empty[STAGES], acc_full[2], acc_empty[2];
+  uint64_t full[MAX_STAGES], empty[MAX_STAGES], acc_full[MAX_ACC], acc_empty[MAX_ACC];
   uint32_t tmem_base;
   int abort;
-  __align__(16) float rn_col[EPI_WARPS][HALF];   // inverse norms of this warp's columns
+  __align__(16) float rn_col[EPI_WARPS][128];    // inverse norms of this warp's columns
 };
 
 enum { MODE_GRAM = 0, MODE_ASSIGN = 1, MODE_SPREAD = 2 };
 
 // The largest-distance pass needs every unordered pair once: tiles that lie wholly below the diagonal
 // are left out (by the producer, the MMA issuer and the epilogue alike).
-template <int MODE> __device__ __forceinline__ bool tile_wanted(int tmi, int tni) {
+template <int MODE, int BN> __device__ __forceinline__ bool tile_wanted(int tmi, int tni) {
   return MODE != MODE_SPREAD || (tni + 1) * BN > tmi * BM;
+}
+
+// Tile `t` of the pass -> block row and block column.  The all-pairs pass walks the nb (nb + 1) / 2
+// blocks with column >= row, row by row; the other passes walk the full grid.
+template <int MODE> __device__ __forceinline__ int tile_count(int ntm, int ntn) {
+  return MODE == MODE_GRAM ? ntm * (ntm + 1) / 2 : ntm * ntn;
+}
+template <int MODE> __device__ __forceinline__ void tile_at(int t, int ntm, int ntn, int &tmi, int &tni) {
+  if (MODE == MODE_GRAM) {
+    // row i starts at i * ntm - i (i - 1) / 2
+    const float b = 2.f * (float)ntm + 1.f;
+    int i = (int)((b - sqrtf(fmaxf(b * b - 8.f * (float)t, 0.f))) * 0.5f);
+    i = max(0, min(i, ntm - 1));
+    while (i > 0 && i * ntm - i * (i - 1) / 2 > t) --i;
+    while (i + 1 < ntm && (i + 1) * ntm - (i + 1) * i / 2 <= t) ++i;
+    tmi = i;
+    tni = i + (t - (i * ntm - i * (i - 1) / 2));
+  } else {
+    tmi = t / ntn;
+    tni = t % ntn;
+  }
 }
 
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -113,11 +146,15 @@ __device__ __forceinline__ float ex2_approx(float x) {
 // One 32-column chunk of the epilogue of the all-pairs pass for one row (= one lane): distance
 // (Eq. 5), density term (Eq. 6) as an integer multiple of 2^-30, adjacency bit d <= d_c, band count.
 // EDGE adds the per-element checks that only edge chunks need (diagonal, columns past the end).
-// The arithmetic is that of DistF (common.cuh) written out so that three terms are summed in 32 bits.
-template <bool EDGE>
+// COLS (blocks above the diagonal) also hands every pair to its column: the warp's 32 x 32 terms go
+// through a shared-memory buffer `tr` (row stride 36 words: conflict-free stores, 16-byte loads), lane k
+// adds the 32 terms of column k, and a 32 x 32 bit transpose gives it the column's adjacency word.  The arithmetic is that of DistF (common.cuh) with the two inverse norms multiplied first,
+// written out so that three terms are summed in 32 bits.
+template <bool EDGE, bool COLS>
 __device__ __forceinline__ void gram_chunk(const uint32_t (&v)[32], const float *rn_col, float rni, int row, int c0,
-                                           int ncols, float d_c, float neg_k, unsigned long long &rowsum,
-                                           uint32_t &bits, int &band) {
+                                           int ncols, float d_c, float neg_k, int lane, uint32_t *tr,
+                                           unsigned long long &rowsum, uint32_t &bits, int &band,
+                                           unsigned long long &colsum, uint32_t &colbits) {
   uint32_t b = 0u;
   unsigned long long s = 0ull;
   uint32_t s3 = 0u;                                 // three terms, each at most 2^30, fit in 32 bits
@@ -129,42 +166,74 @@ __device__ __forceinline__ void gram_chunk(const uint32_t (&v)[32], const float 
 #pragma unroll
     for (int kk = 0; kk < 4; ++kk) {
       const int k = k4 + kk;
-      float dd = DistF::dist(__uint_as_float(v[k]), rni, rnj[kk]);
+      // rn_i * rn_j first: a pair must get the same distance whichever of the two is the row, so that
+      // duplicate keys keep exactly equal densities
+      float dd = fminf(fmaxf(1.0f - __uint_as_float(v[k]) * (rni * rnj[kk]), 0.0f), 2.0f);
       bool ok = true;
       if (EDGE) {
         const int gj = c0 + k;
         if (gj == row) dd = 0.f;
         ok = gj < ncols;
       }
-      const uint32_t term = __float2uint_rn(ex2_approx(dd * neg_k) * (float)(1u << kRhoShift));
-      const bool within = dd <= d_c;
+      uint32_t term = __float2uint_rn(ex2_approx(dd * neg_k) * (float)(1u << kRhoShift));
+      bool within = dd <= d_c;
       const bool inband = fabsf(dd - d_c) <= 1e-6f;
       if (EDGE) {
-        if (ok) {
-          s3 += term;
-          if (within) b |= 1u << k;
-          if (inband && row < c0 + k) ++bnd;
-        }
+        if (!ok) { term = 0u; within = false; }
+        if (ok && inband && row < c0 + k) ++bnd;
       } else {
-        s3 += term;
-        if (within) b |= 1u << k;
         if (inband) ++bnd;
       }
+      s3 += term;
+      if (within) b |= 1u << k;
       if (k % 3 == 2 || k == 31) { s += s3; s3 = 0u; }   // a run of keys at distance 0 adds 2^30 each
+      if (COLS) tr[k * 36 + lane] = term;
     }
   }
   rowsum += s;
   bits = b;
   band += bnd;
+  if (COLS) {
+    __syncwarp();
+    // lane k: the 32 terms of column k, three to a 32-bit partial sum as above
+    unsigned long long cs = 0ull;
+    uint32_t c3 = 0u;
+    const uint4 *src = reinterpret_cast<const uint4 *>(tr + lane * 36);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const uint4 x = src[j];
+      const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        c3 += xs[i];
+        if ((j * 4 + i) % 3 == 2 || j * 4 + i == 31) { cs += c3; c3 = 0u; }
+      }
+    }
+    colsum = cs;
+    // transpose the 32 x 32 bit matrix (lane l holds row l): five exchange steps
+    uint32_t w = b;
+#pragma unroll
+    for (int sft = 16; sft >= 1; sft >>= 1) {
+      const uint32_t m = sft == 16 ? 0x0000FFFFu : sft == 8 ? 0x00FF00FFu : sft == 4 ? 0x0F0F0F0Fu
+                         : sft == 2 ? 0x33333333u : 0x55555555u;
+      const uint32_t y = __shfl_xor_sync(0xffffffffu, w, sft);
+      w = (lane & sft) ? ((w & ~m) | ((y >> sft) & m)) : ((w & m) | ((y << sft) & ~m));
+    }
+    colbits = w;
+    __syncwarp();                                   // tr may be rewritten by the next chunk
+  }
 }
 
 }  // namespace
 
-// grid (X, B), 320 threads, dynamic smem = 1024 (alignment slack) + STAGES * STAGE_BYTES.
+// grid (X, B), 320 threads, dynamic smem = TileCfg<BN>::SMEM.
 // kept_rows (assignment only): rows are the gathered survivors (Kp, rnk) instead of all tokens.
-template <int MODE>
+template <int MODE, int BN>
 __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant__ Batch bt,
                                                            const __grid_constant__ TmapSet tm, int kept_rows) {
+  using Cfg = TileCfg<BN>;
+  constexpr int STAGES = Cfg::STAGES, NACC = Cfg::NACC, HALF = Cfg::HALF;
+  constexpr int STAGE_BYTES = Cfg::STAGE_BYTES, B_BYTES = Cfg::B_BYTES;
   const ImgDesc &im = bt.img[blockIdx.y];
   TL_SCOPE(im, MODE == MODE_GRAM ? 4 : 6);
   (void)kept_rows;
@@ -178,13 +247,13 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
   else if (MODE == MODE_SPREAD) { nrows = im.N; ncols = im.N; }
   else { nrows = kept_rows ? *im.q_ptr : im.N; ncols = *im.C_ptr; }
   const int ntm = (nrows + BM - 1) / BM, ntn = (ncols + BN - 1) / BN;
-  const int ntiles = ntm * ntn;
+  const int ntiles = tile_count<MODE>(ntm, ntn);
   if ((int)blockIdx.x >= ntiles) return;            // uniform: nothing allocated yet
   const int nslab = bt.d_k / BK;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(&sh.acc_full[a], 1); mbar_init(&sh.acc_empty[a], EPI_WARPS); }
+    for (int a = 0; a < NACC; ++a) { mbar_init(&sh.acc_full[a], 1); mbar_init(&sh.acc_empty[a], EPI_WARPS); }
     sh.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -201,8 +270,9 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
       uint32_t it = 0;
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < ntiles; tile += gridDim.x) {
-        const int tmi = tile / ntn, tni = tile % ntn;
-        if (!tile_wanted<MODE>(tmi, tni)) continue;
+        int tmi, tni;
+        tile_at<MODE>(tile, ntm, ntn, tmi, tni);
+        if (!tile_wanted<MODE, BN>(tmi, tni)) continue;
         for (int ks = 0; ks < nslab; ++ks, ++it) {
           const int s = it % STAGES;
           if (!mbar_wait(&sh.empty[s], ((it / STAGES) & 1) ^ 1)) { ok = false; break; }
@@ -210,7 +280,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
           mbar_arrive_expect_tx(&sh.full[s], STAGE_BYTES);
           tma_load_2d(a_dst, ma, &sh.full[s], ks * BK, tmi * BM);
           tma_load_2d(b_dst, mb, &sh.full[s], ks * BK, tni * BN);
-          tma_load_2d(b_dst + B_BYTES / 2, mb, &sh.full[s], ks * BK, tni * BN + BN / 2);
+          if (BN == 256) tma_load_2d(b_dst + B_BYTES / 2, mb, &sh.full[s], ks * BK, tni * BN + BN / 2);
         }
       }
       if (!ok) atomicExch(&sh.abort, 1);
@@ -227,9 +297,11 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
       uint32_t it = 0, tcount = 0;
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < ntiles; tile += gridDim.x) {
-        if (!tile_wanted<MODE>(tile / ntn, tile % ntn)) continue;
-        const uint32_t a = tcount & 1;
-        if (!mbar_wait(&sh.acc_empty[a], ((tcount >> 1) & 1) ^ 1)) { ok = false; break; }
+        int tmi, tni;
+        tile_at<MODE>(tile, ntm, ntn, tmi, tni);
+        if (!tile_wanted<MODE, BN>(tmi, tni)) continue;
+        const uint32_t a = tcount % NACC;
+        if (!mbar_wait(&sh.acc_empty[a], ((tcount / NACC) & 1) ^ 1)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + a * BN;
         for (int ks = 0; ks < nslab; ++ks, ++it) {
@@ -239,7 +311,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
           const uint32_t a_addr = smem_u32(ring + (size_t)s * STAGE_BYTES), b_addr = a_addr + A_BYTES;
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k)
-            umma_bf16(d_tmem, smem_desc(a_addr + k * 32), smem_desc(b_addr + k * 32), kIdesc, (ks | k) != 0);
+            umma_bf16(d_tmem, smem_desc(a_addr + k * 32), smem_desc(b_addr + k * 32), Cfg::IDESC, (ks | k) != 0);
           umma_commit(&sh.empty[s]);               // frees the slab once these MMAs have read it
         }
         if (ok) umma_commit(&sh.acc_full[a]);      // accumulator complete
@@ -253,14 +325,16 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
     const int qd = warp & 3;                        // tensor-memory lane quadrant this warp may read
     const int half = ew >> 2;                       // which half of the tile's columns
     float *rn_col = sh.rn_col[ew];
+    uint32_t *tr = reinterpret_cast<uint32_t *>(ring + Cfg::RING - 1024) + ew * (32 * 36);   // BN = 128 only
     uint32_t tcount = 0;
     int band = 0;
     bool ok = true;
     float mx = 0.f;                                 // largest distance seen by this lane (MODE_SPREAD)
     for (int tile = blockIdx.x; ok && tile < ntiles; tile += gridDim.x) {
-      const int tmi = tile / ntn, tni = tile % ntn;
-      if (!tile_wanted<MODE>(tmi, tni)) continue;
-      const uint32_t a = tcount & 1;
+      int tmi, tni;
+      tile_at<MODE>(tile, ntm, ntn, tmi, tni);
+      if (!tile_wanted<MODE, BN>(tmi, tni)) continue;
+      const uint32_t a = tcount % NACC;
       const int cbase = tni * BN + half * HALF;     // first column of this warp
       // inverse norms of this warp's columns and of this lane's row (in flight while the MMAs run)
       const float *rn_src = MODE == MODE_GRAM ? im.rnk : (MODE == MODE_SPREAD ? im.rn : im.rnc);
@@ -275,11 +349,21 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
       const int row = tmi * BM + qd * 32 + lane;
       const bool row_ok = row < nrows;
       const bool kept_space = MODE == MODE_GRAM || (MODE == MODE_ASSIGN && kept_rows);
-      const float rni = row_ok ? (kept_space ? im.rnk[row] : im.rn[row]) : 0.f;
+      float rni = row_ok ? (kept_space ? im.rnk[row] : im.rn[row]) : 0.f;
+      if (MODE == MODE_GRAM) {
+        // the all-pairs pass multiplies the two inverse norms first; a vanishing key (inverse norm at
+        // its clamp, 1e20) takes 0 here so that the product stays finite: dot product 0, distance 1
+        constexpr float kHuge = 1e19f;
+        if (rni > kHuge) rni = 0.f;
+        if (r4.x > kHuge) r4.x = 0.f;
+        if (r4.y > kHuge) r4.y = 0.f;
+        if (r4.z > kHuge) r4.z = 0.f;
+        if (r4.w > kHuge) r4.w = 0.f;
+      }
       __syncwarp();
-      reinterpret_cast<float4 *>(rn_col)[lane] = r4;
+      if (lane * 4 < HALF) reinterpret_cast<float4 *>(rn_col)[lane] = r4;
       __syncwarp();
-      if (!mbar_wait_warp(&sh.acc_full[a], (tcount >> 1) & 1)) { ok = false; break; }
+      if (!mbar_wait_warp(&sh.acc_full[a], (tcount / NACC) & 1)) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + a * BN + half * HALF + ((uint32_t)(qd * 32) << 16);
       unsigned long long rowsum = 0ull;
@@ -287,6 +371,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
       int bi = 0;
       const float d_c = im.d_c, neg_k = -im.inv_dn_log2e;
       const int r0 = tmi * BM + qd * 32;
+      const bool above = MODE == MODE_GRAM && tni > tmi;   // block above the diagonal: rows and columns
 #pragma unroll 1
       for (int ch = 0; ch < HALF / 32; ++ch) {
         const int c0 = cbase + ch * 32;
@@ -295,13 +380,30 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
         tmem_ld32(taddr + ch * 32, v);
         tmem_ld_wait();
         if (MODE == MODE_GRAM) {
-          uint32_t bits;
-          const bool edge = (c0 + 32 > ncols) || (c0 < r0 + 32 && c0 + 32 > r0);
-          if (edge) gram_chunk<true>(v, rn_col + ch * 32, rni, row, c0, ncols, d_c, neg_k, rowsum, bits, band);
-          else {
+          uint32_t bits, colbits = 0u;
+          unsigned long long colsum = 0ull;
+          if (above) {
+            // every row of this block is a survivor (only the last block row is ragged, and it has no
+            // block to its right); each pair (row, column) is also the pair (column, row)
             int bnd = 0;
-            gram_chunk<false>(v, rn_col + ch * 32, rni, row, c0, ncols, d_c, neg_k, rowsum, bits, bnd);
-            if (row < c0) band += bnd;              // each unordered pair once; the chunk lies wholly on one side
+            if (c0 + 32 > ncols)
+              gram_chunk<true, true>(v, rn_col + ch * 32, rni, row, c0, ncols, d_c, neg_k, lane, tr, rowsum, bits, bnd, colsum, colbits);
+            else
+              gram_chunk<false, true>(v, rn_col + ch * 32, rni, row, c0, ncols, d_c, neg_k, lane, tr, rowsum, bits, bnd, colsum, colbits);
+            band += bnd;                            // row < column throughout
+            const int gj = c0 + lane;
+            if (gj < ncols) {
+              atomicAdd(&im.rho_fix[gj], colsum);
+              im.adj[(size_t)gj * im.Wp + (r0 >> 5)] = colbits;
+            }
+          } else {
+            const bool edge = (c0 + 32 > ncols) || (c0 < r0 + 32 && c0 + 32 > r0);
+            if (edge) gram_chunk<true, false>(v, rn_col + ch * 32, rni, row, c0, ncols, d_c, neg_k, lane, tr, rowsum, bits, band, colsum, colbits);
+            else {
+              int bnd = 0;
+              gram_chunk<false, false>(v, rn_col + ch * 32, rni, row, c0, ncols, d_c, neg_k, lane, tr, rowsum, bits, bnd, colsum, colbits);
+              if (row < c0) band += bnd;            // each unordered pair once; the chunk lies wholly on one side
+            }
           }
           if (row_ok) im.adj[(size_t)row * im.Wp + (c0 >> 5)] = bits;
         } else if (MODE == MODE_SPREAD) {
@@ -382,7 +484,7 @@ bool encode_rows(CUtensorMap *map, const void *base, long long rows, long long l
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-constexpr size_t kUmmaSmem = 1024 + (size_t)STAGES * STAGE_BYTES;
+constexpr int kGramBN = 128, kWideBN = 256;
 
 }  // namespace
 
@@ -393,17 +495,19 @@ cudaError_t umma_configure() {
   if (e != cudaSuccess) return e;
   if (qres != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
   g_encode = reinterpret_cast<EncodeTiledFn>(fn);
-  e = cudaFuncSetAttribute(k_tiles_umma<MODE_GRAM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kUmmaSmem);
+  e = cudaFuncSetAttribute(k_tiles_umma<MODE_GRAM, kGramBN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)TileCfg<kGramBN>::SMEM);
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(k_tiles_umma<MODE_SPREAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kUmmaSmem);
+  e = cudaFuncSetAttribute(k_tiles_umma<MODE_SPREAD, kWideBN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)TileCfg<kWideBN>::SMEM);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(k_tiles_umma<MODE_ASSIGN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kUmmaSmem);
+  return cudaFuncSetAttribute(k_tiles_umma<MODE_ASSIGN, kWideBN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)TileCfg<kWideBN>::SMEM);
 }
 
 bool umma_supported(int d_k) { return g_encode != nullptr && d_k % BK == 0; }
 
-static int umma_grid_x(int max_rows, int max_cols, int B, int sms) {
-  const long long tiles = (long long)((max_rows + BM - 1) / BM) * ((max_cols + BN - 1) / BN);
+static int umma_grid_x(long long tiles, int B, int sms) {
   long long x = sms / B;                            // one CTA per SM: all CTAs of the batch run at once
   if (x < 1) x = 1;
   if (x > tiles) x = tiles;
@@ -417,8 +521,9 @@ cudaError_t launch_gram_umma(const Batch &bt, int maxN, const ClusterCfg &cfg, c
     if (!encode_rows(&tm.a[b], im.Kp, im.Np, bt.d_k, bt.d_k)) return cudaErrorInvalidValue;
     tm.b[b] = tm.a[b];
   }
-  dim3 grid(umma_grid_x(maxN, maxN, bt.B, cfg.sm_count), bt.B);
-  k_tiles_umma<MODE_GRAM><<<grid, THREADS, kUmmaSmem, st>>>(bt, tm, 0);
+  const long long nb = (maxN + BM - 1) / BM;
+  dim3 grid(umma_grid_x(nb * (nb + 1) / 2, bt.B, cfg.sm_count), bt.B);
+  k_tiles_umma<MODE_GRAM, kGramBN><<<grid, THREADS, TileCfg<kGramBN>::SMEM, st>>>(bt, tm, 0);
   return cudaGetLastError();
 }
 
@@ -431,8 +536,9 @@ cudaError_t launch_assign_umma(const Batch &bt, int maxN, bool kept_rows, const 
     } else if (!encode_rows(&tm.a[b], im.Kc, im.N, im.ldKc, bt.d_k)) return cudaErrorInvalidValue;
     if (!encode_rows(&tm.b[b], im.Kcen, im.Np, bt.d_k, bt.d_k)) return cudaErrorInvalidValue;
   }
-  dim3 grid(umma_grid_x(maxN, maxN, bt.B, cfg.sm_count), bt.B);
-  k_tiles_umma<MODE_ASSIGN><<<grid, THREADS, kUmmaSmem, st>>>(bt, tm, kept_rows ? 1 : 0);
+  const long long tiles = (long long)((maxN + BM - 1) / BM) * ((maxN + kWideBN - 1) / kWideBN);
+  dim3 grid(umma_grid_x(tiles, bt.B, cfg.sm_count), bt.B);
+  k_tiles_umma<MODE_ASSIGN, kWideBN><<<grid, THREADS, TileCfg<kWideBN>::SMEM, st>>>(bt, tm, kept_rows ? 1 : 0);
   return cudaGetLastError();
 }
 
@@ -444,8 +550,9 @@ cudaError_t launch_spread_umma(const Batch &bt, int maxN, const ClusterCfg &cfg,
     if (!encode_rows(&tm.a[b], im.Kc, im.N, im.ldKc, bt.d_k)) return cudaErrorInvalidValue;
     tm.b[b] = tm.a[b];
   }
-  dim3 grid(umma_grid_x(maxN, maxN, bt.B, cfg.sm_count), bt.B);
-  k_tiles_umma<MODE_SPREAD><<<grid, THREADS, kUmmaSmem, st>>>(bt, tm, 0);
+  const long long tiles = (long long)((maxN + BM - 1) / BM) * ((maxN + kWideBN - 1) / kWideBN);
+  dim3 grid(umma_grid_x(tiles, bt.B, cfg.sm_count), bt.B);
+  k_tiles_umma<MODE_SPREAD, kWideBN><<<grid, THREADS, TileCfg<kWideBN>::SMEM, st>>>(bt, tm, 0);
   return cudaGetLastError();
 }
 
