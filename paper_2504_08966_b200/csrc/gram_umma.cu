@@ -29,6 +29,9 @@ constexpr int BK = 64;            // bf16 elements per K-slab = one 128-byte swi
 constexpr int A_BYTES = BM * BK * 2;
 constexpr int TMEM_COLS = 512;    // all of an SM's tensor memory
 constexpr int MAX_STAGES = 6;
+constexpr int EPI_WARPS = 8;      // per tensor-memory lane quadrant EPI_WARPS / 4 warps share the columns
+                                  // (16 measured the same on the all-pairs pass and slower on the others)
+constexpr int THREADS = 64 + EPI_WARPS * 32;
 constexpr int MAX_ACC = 4;
 
 // Per tile width BN (UMMA N): 256 columns for the rows x centres and the largest-distance passes,
@@ -38,10 +41,10 @@ template <int BN> struct TileCfg {
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int STAGES = BN == 256 ? 4 : 5;
   static constexpr int NACC = TMEM_COLS / BN;      // accumulators in tensor memory
-  static constexpr int HALF = BN / 2;              // columns per epilogue warp
+  static constexpr int HALF = BN / (EPI_WARPS / 4); // columns per epilogue warp
   // BN = 128 (all-pairs pass): one 32 x 32 exchange buffer per epilogue warp behind the ring
   static constexpr size_t RING = 1024 + (size_t)STAGES * STAGE_BYTES;
-  static constexpr size_t SMEM = RING + (BN == 128 ? (size_t)8 * 32 * 36 * 4 : 0);
+  static constexpr size_t SMEM = RING + (BN == 128 ? (size_t)EPI_WARPS * 32 * 36 * 4 : 0);
   // kind::f16 instruction descriptor: fp32 accumulate, bf16 x bf16, both operands K-major.
   static constexpr uint32_t IDESC =
       (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
@@ -98,8 +101,6 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
   return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
          ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
 }
-constexpr int EPI_WARPS = 8;      // two per tensor-memory lane quadrant; each takes half of the columns
-constexpr int THREADS = 64 + EPI_WARPS * 32;
 
 struct Shared {
   uint64_t full[MAX_STAGES], empty[MAX_STAGES], acc_full[MAX_ACC], acc_empty[MAX_ACC];
