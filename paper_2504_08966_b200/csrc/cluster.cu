@@ -300,32 +300,28 @@ __global__ void __launch_bounds__(256) k_centers(const __grid_constant__ Batch b
   constexpr int V = Vec<T>::N;
   cooperative_groups::grid_group grid = cooperative_groups::this_grid();
   TL_SCOPE(bt.img[0], 5);
-  extern __shared__ unsigned long long skeys[];          // [keys_cap] densities of the current image
+  extern __shared__ unsigned long long skeys[];          // [keys_cap] densities of this CTA's image
   const int lane = threadIdx.x & 31;
-  const int nwarps = gridDim.x * 8;
-  const int gw = blockIdx.x * 8 + (threadIdx.x >> 5);
-  int qs[kMaxBatchPerLaunch + 1];
-  qs[0] = 0;
-  for (int b = 0; b < bt.B; ++b) qs[b + 1] = qs[b] + *bt.img[b].q_ptr;
-  const int total = qs[bt.B];
+  // The CTAs are shared out evenly among the images (the last image also takes the remainder); a CTA
+  // works on one image throughout, so the images of a batch are resolved side by side.
+  const int per = gridDim.x / bt.B;
+  const int b = min((int)blockIdx.x / per, bt.B - 1);
+  const int ncta = b == bt.B - 1 ? (int)gridDim.x - per * (bt.B - 1) : per;
+  const int nwarps = ncta * 8;
+  const int gw = ((int)blockIdx.x - b * per) * 8 + (threadIdx.x >> 5);
+  const ImgDesc &im = bt.img[b];
+  const int q = *im.q_ptr, nw = (q + 31) >> 5;
 
   // part 1: keep only the neighbours that come earlier in density order
   uint32_t cached[kAdjRegs];
   int cached_item = -1;
-  for (int b = 0; b < bt.B; ++b) {
-    const ImgDesc &im = bt.img[b];
-    const int q = qs[b + 1] - qs[b], nw = (q + 31) >> 5;
+  {
     const bool in_smem = q <= keys_cap;
-    __syncthreads();
     if (in_smem)
       for (int r = threadIdx.x; r < q; r += 256) skeys[r] = im.rho_fix[r];
     __syncthreads();
     const unsigned long long *keys = in_smem ? skeys : im.rho_fix;
-    // first item of this warp that lies in image b
-    int item = gw;
-    if (item < qs[b]) item += ((qs[b] - item + nwarps - 1) / nwarps) * nwarps;
-    for (; item < qs[b + 1]; item += nwarps) {
-      const int r = item - qs[b];
+    for (int r = gw; r < q; r += nwarps) {
       const unsigned long long mine = keys[r];
       uint32_t *row = im.adj + (size_t)r * im.Wp;
       const bool keep_regs = cached_item < 0 && nw <= 32 * kAdjRegs;
@@ -357,7 +353,7 @@ __global__ void __launch_bounds__(256) k_centers(const __grid_constant__ Batch b
         }
         row[wd] = out;
       }
-      if (keep_regs) cached_item = item;
+      if (keep_regs) cached_item = r;
       if (lane == 0) {
         const float rf = (float)((double)mine * (1.0 / (double)(1u << kRhoShift)));
         im.rho[r] = rf;
@@ -374,14 +370,10 @@ __global__ void __launch_bounds__(256) k_centers(const __grid_constant__ Batch b
   while (pending && sweeps < kSpinLimit) {
     pending = 0;
     ++sweeps;
-    for (int item = gw; item < total; item += nwarps) {
-      int b = 0;
-      while (item >= qs[b + 1]) ++b;
-      const ImgDesc &im = bt.img[b];
-      const int r = item - qs[b], q = qs[b + 1] - qs[b], nw = (q + 31) >> 5;
+    for (int r = gw; r < q; r += nwarps) {
       const uint32_t mybit = 1u << (r & 31);
       bool hit_center = false, alive = false;
-      if (item == cached_item) {                  // the masked adjacency of this row is in registers
+      if (r == cached_item) {                     // the masked adjacency of this row is in registers
         if (cached_done) continue;
         uint32_t cm[kAdjRegs], rm[kAdjRegs];
 #pragma unroll
@@ -411,21 +403,19 @@ __global__ void __launch_bounds__(256) k_centers(const __grid_constant__ Batch b
       alive = __any_sync(0xffffffffu, alive);
       if (hit_center) {
         if (lane == 0) atomicOr(&im.rmask[r >> 5], mybit);
-        if (item == cached_item) cached_done = true;
+        if (r == cached_item) cached_done = true;
       } else if (!alive) {
         if (lane == 0) atomicOr(&im.cmask[r >> 5], mybit);
-        if (item == cached_item) cached_done = true;
+        if (r == cached_item) cached_done = true;
       } else {
         pending = 1;
       }
     }
     if (pending) __nanosleep(100);                 // the masks are polled by thousands of warps: do not hammer them
   }
-  if (lane == 0 && total > 0) {
-    for (int b = 0; b < bt.B; ++b) {
-      if (pending) atomicMin(&bt.img[b].cnt[PACT_CNT_STATUS], (int)PACT_ERR_TIMEOUT);
-      atomicMax(&bt.img[b].cnt[PACT_CNT_SWEEPS], sweeps);
-    }
+  if (lane == 0 && gw < q) {
+    if (pending) atomicMin(&im.cnt[PACT_CNT_STATUS], (int)PACT_ERR_TIMEOUT);
+    atomicMax(&im.cnt[PACT_CNT_SWEEPS], sweeps);
   }
 
   // part 3: every decision is final once all CTAs are here
@@ -439,9 +429,7 @@ __global__ void __launch_bounds__(256) k_centers(const __grid_constant__ Batch b
   // from global memory.
   __shared__ int wsum3[8];
   __shared__ int s_carry3;
-  for (int b = 0; b < bt.B; ++b) {
-    const ImgDesc &im = bt.img[b];
-    const int q = qs[b + 1] - qs[b], nw = (q + 31) >> 5;
+  {
     const bool staged = q <= keys_cap;              // nw words and nw counts fit where the densities were
     uint32_t *cm = reinterpret_cast<uint32_t *>(skeys);
     int *pref = reinterpret_cast<int *>(skeys) + nw;
@@ -469,10 +457,7 @@ __global__ void __launch_bounds__(256) k_centers(const __grid_constant__ Batch b
         __syncthreads();
       }
     }
-    int item = gw;
-    if (item < qs[b]) item += ((qs[b] - item + nwarps - 1) / nwarps) * nwarps;
-    for (; item < qs[b + 1]; item += nwarps) {
-      const int r = item - qs[b];
+    for (int r = gw; r < q; r += nwarps) {
       int c, all;
       bool is_center;
       if (staged) {
