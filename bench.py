@@ -33,7 +33,7 @@ N_COPIES = 4          # input copies rotated between steps so that no step finds
 NCU_TRAFFIC: dict = {
     ("single_image", "merge"): 52311808 + 444160,
     ("single_image", "prepass"): 67235328 + 396800,
-    ("single_image", "gram_density"): 4024064,
+    ("single_image", "gram_density"): 3915520,
     ("single_image", "assign"): 8372224,
 }
 
