@@ -305,7 +305,7 @@ k_merge(const __grid_constant__ Batch bt) {
         }
       }
     }
-    const float fs = center_only ? 1.0f : (float)size;
+    const float inv = center_only ? 1.0f : 1.0f / (float)size;   // one division per unit, not one per element
     if (nch > 1) {
       // scratch rows: the clusters that are summed in several chunks take theirs in cluster order
       int base = 0;
@@ -352,7 +352,7 @@ k_merge(const __grid_constant__ Batch bt) {
       if (g < ng) {
         float y[8];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) y[e] = acc[v][e] / fs;
+        for (int e = 0; e < 8; ++e) y[e] = acc[v][e] * inv;
         store_vec8<O>(Ho + (size_t)dst * im.ldHo + g * 8, y);
       }
     }

@@ -232,6 +232,40 @@ def test_graph_replay_matches_direct_call_bitwise():
     g.close()
 
 
+def test_contexts_on_separate_streams_do_not_interfere():
+    """Independent requests in flight at once: one context, workspace and graph per stream; every
+    stream must reproduce what the same request gives alone."""
+    from paper_2504_08966_b200 import binding as pb
+    wls = [workloads.single_image(seed=70 + i, N=1800 + 211 * i, T=10, n_blobs=40) for i in range(3)]
+    alone = []
+    for wl in wls:
+        outs, _ = gpu_reduce(wl, torch.bfloat16)
+        alone.append(outs[0])
+    ctxs, graphs, ims, streams = [], [], [], []
+    for wl in wls:
+        ctx = pb.Context(wl.d, wl.n_qh, wl.n_kvh, wl.d_h, wl.dtype, torch.bfloat16)
+        im = pb.device_image(wl.images[0], torch.bfloat16)
+        ctxs.append(ctx)
+        ims.append(im)
+        graphs.append(ctx.pact_graph_create([im], pb.make_params(lam=wl.lam, d_c=wl.d_c, d_n=wl.d_n, alpha=wl.alpha)))
+        streams.append(torch.cuda.Stream())
+    torch.cuda.synchronize()
+    for rep in range(20):
+        for g, st in zip(graphs, streams):
+            with torch.cuda.stream(st):
+                g.launch()
+    torch.cuda.synchronize()
+    for im, ref in zip(ims, alone):
+        cnt = im.counters.cpu().numpy()
+        n_out = int(cnt[pb.CNT["n_out"]])
+        assert int(cnt[pb.CNT["status"]]) == 0 and n_out == ref["n_out"]
+        assert np.array_equal(im.label.cpu().numpy(), ref["label"])
+        assert torch.equal(im.H_out[:n_out].cpu().view(torch.int16), ref["H_out_raw"].view(torch.int16))
+        assert np.array_equal(im.P_out[:n_out].cpu().numpy(), ref["P_out"])
+    for g in graphs:
+        g.close()
+
+
 # ------------------------------------------------------------------ stage calls against the oracle's stages
 
 @pytest.fixture(scope="module")
