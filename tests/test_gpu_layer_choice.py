@@ -67,6 +67,14 @@ def test_spread_fp32_keys_and_more_layers_than_one_launch_takes():
     assert layer == 35 == orc.select_layer([f64(K) for K in late], 0.2)
 
 
+def test_spread_bf16_keys_of_a_width_the_tensor_core_tiles_do_not_take():
+    layers = workloads.layer_keys(seed=14, n_layers=5, N=333, n_h=3, d_h=32)
+    want = _oracle(layers)
+    got, layer = _run(layers, 0.05, torch.bfloat16, 3, 32)
+    assert np.abs(got - want).max() <= _tolerance(96)
+    assert layer == orc.select_layer([f64(K) for K in layers], 0.05)
+
+
 def test_spread_special_cases():
     row = torch.from_numpy(np.random.default_rng(3).standard_normal((1, 512))).to(torch.bfloat16)
     same = (row.float() * torch.tensor([[1.0], [2.0], [0.5], [4.0]])).to(torch.bfloat16)   # exact multiples

@@ -133,6 +133,8 @@ def test_no_text_tokens_and_gqa_and_distinct_clustering_keys():
     _check_workload(_small(seed=42, n_qh=4), torch.bfloat16)
     _check_workload(_small(seed=43, distinct_k_clu=True), torch.bfloat16)
     _check_workload(_small(seed=44, dtype=torch.float32, d_h=16, n_h=3, d=136), torch.float32)
+    # bf16 keys whose width is not a multiple of 64 take the SIMT tile kernels
+    _check_workload(_small(seed=45, d_h=48, n_h=2, d=264), torch.bfloat16)
 
 
 def test_exact_duplicates_tie_break():
@@ -230,6 +232,36 @@ def test_graph_replay_matches_direct_call_bitwise():
     o = oracle_image(wl, wl.images[0])
     assert np.array_equal(direct[0]["label"], o["label"])
     g.close()
+
+
+def test_full_size_image_as_the_benchmark_runs_it():
+    """The timed configuration: N = 7290, bf16 output, graph replays rotating over input copies."""
+    from paper_2504_08966_b200 import binding as pb
+    wl = workloads.single_image()
+    img = wl.images[0]
+    o = oracle_image(wl, img)
+    ctx = pb.Context(wl.d, wl.n_qh, wl.n_kvh, wl.d_h, wl.dtype, torch.bfloat16)
+    params = pb.make_params(lam=wl.lam, d_c=wl.d_c, d_n=wl.d_n, alpha=wl.alpha)
+    sets = [[pb.device_image(img, torch.bfloat16)] for _ in range(3)]
+    graphs = [ctx.pact_graph_create(ims, params) for ims in sets]
+    for i in range(31):
+        graphs[i % 3].launch()
+    torch.cuda.synchronize()
+    for ims in sets:
+        im = ims[0]
+        cnt = im.counters.cpu().numpy()
+        n_out = int(cnt[pb.CNT["n_out"]])
+        g = {"counters": cnt, "n_out": n_out, "q": int(cnt[pb.CNT["q"]]), "C": int(cnt[pb.CNT["C"]]),
+             "r": int(cnt[pb.CNT["r"]]), "discarded": int(cnt[pb.CNT["discarded"]]),
+             "status": int(cnt[pb.CNT["status"]]), "label": im.label.cpu().numpy(),
+             "keep": im.keep.cpu().numpy().astype(bool), "score": im.score.cpu().numpy(),
+             "H_out": im.H_out[:n_out].to(torch.float64).cpu().numpy(),
+             "P_out": im.P_out[:n_out].cpu().numpy(), "size_out": im.size_out[:n_out].cpu().numpy(),
+             "logw_out": im.logw_out[:n_out].cpu().numpy().astype(np.float64)}
+        assert g["status"] == 0
+        assert not compare_image(o, g, img, True)
+    for gr in graphs:
+        gr.close()
 
 
 def test_contexts_on_separate_streams_do_not_interfere():
