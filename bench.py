@@ -287,6 +287,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="pact", choices=["pact", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--in-flight", type=int, default=4,
+                    help="also report the throughput with this many independent single-image requests in flight")
     ap.add_argument("--workload", default="single_image",
                     choices=["single_image", "video", "batched", "stress", *STAGE_WORKLOADS])
     args = ap.parse_args()
@@ -382,6 +384,37 @@ def main():
     torch.cuda.synchronize()
     plain_ms = e0.elapsed_time(e1) / n_plain
 
+    # ---- independent requests in flight at once: one context, workspace, graph and stream each -----
+    in_flight = None
+    if B == 1 and args.in_flight > 1:
+        S = min(args.in_flight, copies)
+        ctxs = [pb.Context(wl.d, wl.n_qh, wl.n_kvh, wl.d_h, wl.dtype, torch.bfloat16) for _ in range(S)]
+        for c in ctxs:
+            c.ensure_workspace(B, max(im.N for im in wl.images))
+        sgraphs = [ctxs[s].pact_graph_create(sets[s], params) for s in range(S)]
+        streams = [torch.cuda.Stream() for _ in range(S)]
+        n_fl = max(S * 5, min(args.steps, 2000))
+        for rep in range(2):                       # the first pass warms up
+            torch.cuda.synchronize()
+            e0.record()
+            for st in streams:
+                st.wait_event(e0)
+            for i in range(n_fl):
+                with torch.cuda.stream(streams[i % S]):
+                    sgraphs[i % S].launch()
+            for st in streams:
+                ev = torch.cuda.Event()
+                ev.record(st)
+                torch.cuda.current_stream().wait_event(ev)
+            e1.record()
+            torch.cuda.synchronize()
+        fl_ms = e0.elapsed_time(e1) / n_fl
+        ok = all(int(sets[s][0].counters.cpu()[pb.CNT["status"]]) == 0 for s in range(S))
+        in_flight = {"streams": S, "ms_per_step": fl_ms, "value": n_vis / (fl_ms * 1e-3), "unit": UNIT,
+                     "status_ok": ok, "scope": "this GPU"}
+        for g in sgraphs:
+            g.close()
+
     # ---- per-kernel times (separate pass, cold L2 per step via the rotating inputs) ---------
     ctx.profile_enable(True)
     acc: dict = {}
@@ -474,6 +507,7 @@ def main():
                        "l2": f"{copies} input copies rotated between steps ({in_bytes * copies / 1e6:.0f} MB > 126 MB L2)"
                              + ("; per-kernel pass also writes a 512 MB flush buffer" if flush is not None else "")},
             "latency_us": ms_per_step * 1e3 / B, "stream_launch_ms_per_step": plain_ms,
+            "in_flight": in_flight,
             "counts": {"q": q, "C": Cn, "r": r, "sweeps": int(cnt[pb.CNT["sweeps"]]),
                        "band_dc": int(cnt[pb.CNT["band_dc"]]), "band_adc": int(cnt[pb.CNT["band_adc"]])},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
