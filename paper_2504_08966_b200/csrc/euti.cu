@@ -22,20 +22,21 @@ __device__ __forceinline__ double ld_cg_f64(const double *p) {
   return v;
 }
 
-constexpr int kPreThreads = 512;
+constexpr int kPreThreads = 256;              // two CTAs per SM: one loads while the other reduces
 constexpr int kTokWarps = kPreThreads / 32;   // tokens per CTA of the token part of k_prepass
 constexpr int kQCtasMax = kQPartRows;         // CTAs that reduce Q
 
 // ---- Eq. 1 and the norms -----------------------------------------------------------------------
-// grid (GQ + ceil(maxN / 16), B), 512 threads.
+// grid (GQ + ceil(maxN / 8), B), 256 threads, two CTAs per SM (on batches a third faster than one CTA of
+// 512 threads, whose load and reduce phases leave the memory pipe idle in turn; the same on one image).
 //  CTAs [0, GQ): column sums of a contiguous block of rows of Q; the last of them to finish adds
 //                the GQ partial sums in index order and writes the global query.
-//  other CTAs:   one warp per visual token; every 16-byte load of the token's clustering-key row and
+//  other CTAs:   one warp per visual token (8 tokens per CTA); every 16-byte load of the token's clustering-key row and
 //                hidden-state row is issued before the first is used: |h_i| (double) and 1 / |k_i|.
 // (A variant that streamed the rows through a shared-memory ring with bulk copies measured the same on
 // one image and worse on batches: bulk copies issued row by row complete at about 20 GB/s per SM.)
 template <typename T>
-__global__ void __launch_bounds__(kPreThreads) k_prepass(const __grid_constant__ Batch bt, int GQ) {
+__global__ void __launch_bounds__(kPreThreads, 2) k_prepass(const __grid_constant__ Batch bt, int GQ) {
   using D = typename DistOf<T>::type;
   using rn_t = typename D::rn_t;
   constexpr int V = Vec<T>::N;
