@@ -68,6 +68,22 @@ def test_batch_with_per_image_params_and_mixed_sizes():
         assert not compare_image(o, g, img, True)
 
 
+def test_batch_of_sixteen_with_extreme_size_mix():
+    """Sixteen images from 1 to 4100 tokens in one call: every image has its own share of every grid."""
+    sizes = [1, 4100, 2, 33, 700, 129, 3000, 5, 64, 1023, 257, 31, 2048, 300, 17, 1500]
+    imgs, first = [], None
+    for k, n in enumerate(sizes):
+        w = _small(seed=300 + k, N=n, T=k % 5, n_blobs=max(1, min(30, n // 8 + 1)))
+        first = first or w
+        imgs += w.images
+    wl = workloads.Workload("mix16", imgs, first.d, first.n_qh, first.n_kvh, first.d_h, first.dtype, 0.5, 0.3)
+    outs, _ = gpu_reduce(wl, torch.bfloat16)
+    for img, g in zip(wl.images, outs):
+        o = oracle_image(wl, img)
+        bad = compare_image(o, g, img, True)
+        assert not bad, f"N={img.N}: {bad}"
+
+
 # ------------------------------------------------------------------ edge and degenerate cases
 
 def _small(seed=21, N=700, T=9, **kw):
