@@ -246,6 +246,25 @@ k_merge(const __grid_constant__ Batch bt) {
         const int m0 = k * kChunk, m1 = min(size, m0 + kChunk);
         nm = m1 - m0;
         int carry = 0;
+        if (nblk <= 32) {                           // one warp covers all blocks: no CTA-wide scan
+          if (w == 0) {
+            int s0 = 0, cntb = 0;
+            if (lane < nblk) {
+              const uint16_t *row = im.bstart + (size_t)lane * im.bstride;
+              s0 = row[c];
+              cntb = (int)row[c + 1] - s0;
+            }
+            int x = cntb;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+              const int y = __shfl_up_sync(0xffffffffu, x, o);
+              if (lane >= o) x += y;
+            }
+            const int off = x - cntb;               // list position of this block's first member
+            const int a0 = max(off, m0), a1 = min(off + cntb, m1);
+            for (int m = a0; m < a1; ++m) members[m - m0] = im.blocklist[(size_t)lane * kListBlock + s0 + (m - off)];
+          }
+        } else
         for (int bb0 = 0; bb0 < nblk; bb0 += kMrgThreads) {   // thread = block of the member lists
           const int bb = bb0 + t;
           int s0 = 0, cntb = 0;
