@@ -177,7 +177,7 @@ k_merge(const __grid_constant__ Batch bt) {
   extern __shared__ int chunk_off[];               // [C + 1] first chunk of cluster c
   __shared__ int wsum[kMrgThreads / 32];
   __shared__ int s_carry, s_last;
-  __shared__ int members[kChunk];
+  __shared__ int members2[2][kChunk];              // member lists of the current and the previous unit
   const int C = *im.C_ptr;
   const int n_text = im.n_total - im.N;
   const int d = bt.d, ng = d / 8;
@@ -215,12 +215,15 @@ k_merge(const __grid_constant__ Batch bt) {
   const int nblk = (im.N + kListBlock - 1) / kListBlock;
 
   // units are handed out first come, first served (the order does not change any result)
-  __shared__ int s_next;
-  int u = blockIdx.x;
+  // The member list and the next unit's number alternate between two slots: a thread can be at most one
+  // barrier behind, so the slots of unit n are rewritten (for unit n + 2) only after every thread has
+  // passed the barrier of unit n + 1, i.e. is done with unit n.  One CTA-wide barrier per unit.
+  __shared__ int s_next2[2];
+  int u = blockIdx.x, par = 0;
   while (u < n_units) {
     int c = -1, k = 0, nch = 1, size = 1, nm = 1, dst, ptok;
-    __syncthreads();                               // members, wsum and s_next of the previous unit are consumed
-    if (t == 0) s_next = gridDim.x + atomicAdd(&im.cnt[21], 1);   // needed only after this unit's rows
+    int *members = members2[par];
+    if (t == 0) s_next2[par] = gridDim.x + atomicAdd(&im.cnt[21], 1);   // needed only after this unit's rows
     if (u >= n_chunks) {                           // a text row
       const int tr = u - n_chunks;
       const int src = tr < im.vis_start ? tr : tr + im.N;
@@ -347,7 +350,7 @@ k_merge(const __grid_constant__ Batch bt) {
       __syncthreads();
       if (t == 0) s_last = (atomicAdd(&im.cticket[c], 1) == nch - 1);
       __syncthreads();
-      if (!s_last) { u = s_next; continue; }       // the loop head synchronises before s_last and s_next are rewritten
+      if (!s_last) { u = s_next2[par]; par ^= 1; continue; }
       __threadfence();
       const float *p0 = im.mpart + (size_t)base * d;
 #pragma unroll
@@ -380,7 +383,8 @@ k_merge(const __grid_constant__ Batch bt) {
       im.size_out[dst] = size;
       if (im.logw_out) im.logw_out[dst] = logf((float)size);   // Eq. 11: log of the token weight
     }
-    u = s_next;
+    u = s_next2[par];
+    par ^= 1;
   }
 }
 
