@@ -31,7 +31,7 @@ N_COPIES = 4          # input copies rotated between steps so that no step finds
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
 # (workload, kernel) -> bytes; absent = not captured for the kernel as it stands
 NCU_TRAFFIC: dict = {
-    ("single_image", "merge"): 52308736 + 440576,
+    ("single_image", "merge"): 52310016 + 341248,
     ("single_image", "prepass"): 67227392 + 423936,
     ("single_image", "gram_density"): 3915520,
     ("single_image", "assign"): 8372224,
