@@ -32,6 +32,8 @@
  *  - Percentile(s, lambda): with m = min(floor(lambda*N + 1e-6), N-1) and tau the (m+1)-th
  *    smallest score, a token is important iff s_i >= tau (Eq. 3) - ties at tau are kept.
  *  - The clustering vector of a token is the concatenation of its key heads (width d_k).
+ *  - Distances are clamped to [0, 2]; d_ii = 0; a key whose norm vanishes (below about 1e-19)
+ *    is at distance 1 from every other key.
  *  - Density ties go to the lower token index; a vector becomes a centre iff its distance to
  *    every earlier centre is strictly greater than d_c; argmin ties go to the lower cluster id.
  *  - Cluster ids number the centres by ascending token index; merged rows are emitted in
