@@ -12,9 +12,10 @@
 //               columns each), distance arithmetic of common.cuh
 // Several accumulators (512 / BN of them share the tensor memory) let the epilogue of tile t overlap
 // the MMAs of the next tiles.  The all-pairs pass computes every unordered pair of survivors once: a
-// 128 x 128 block above the diagonal serves its rows (density sums, adjacency words) and, through
-// warp-wide sums and ballots, its columns as well; blocks on the diagonal serve their rows only.  Every mbarrier wait is bounded; when one runs out the CTA raises the image's status
-// word, drains what it armed, frees its tensor memory and returns.
+// 128 x 128 block above the diagonal serves its rows (density sums, adjacency words) and, through a
+// shared-memory exchange of the terms and a warp transpose of the adjacency bits, its columns as well;
+// blocks on the diagonal serve their rows only.  Every mbarrier wait is bounded; when one runs out the
+// CTA raises the image's status word, drains what it armed, frees its tensor memory and returns.
 #include <cuda.h>
 
 #include "kernels.cuh"
