@@ -133,10 +133,23 @@ template <int MODE> __device__ __forceinline__ void tile_at(int t, int ntm, int 
     while (i + 1 < ntm && (i + 1) * ntm - (i + 1) * i / 2 <= t) ++i;
     tmi = i;
     tni = i + (t - (i * ntm - i * (i - 1) / 2));
+  } else if (MODE == MODE_ASSIGN) {
+    // full-width column tiles first, the (usually narrow) last column last: the CTAs that take a second
+    // tile then take a cheap one
+    const int fullc = ntn - 1, nfull = ntm * fullc;
+    if (t < nfull) { tmi = t / fullc; tni = t % fullc; }
+    else { tmi = t - nfull; tni = fullc; }
   } else {
     tmi = t / ntn;
     tni = t % ntn;
   }
+}
+// Columns of tile column tni that the MMA has to produce: the rows x centres pass stops at the last
+// centre, rounded up to the instruction's granularity of 16.
+template <int MODE, int BN> __device__ __forceinline__ int tile_width(int tni, int ncols) {
+  if (MODE != MODE_ASSIGN) return BN;
+  const int left = ncols - tni * BN;
+  return left >= BN ? BN : ((left + 15) & ~15);
 }
 
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -275,14 +288,16 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
         int tmi, tni;
         tile_at<MODE>(tile, ntm, ntn, tmi, tni);
         if (!tile_wanted<MODE, BN>(tmi, tni)) continue;
+        const int bw = tile_width<MODE, BN>(tni, ncols);
         for (int ks = 0; ks < nslab; ++ks, ++it) {
           const int s = it % STAGES;
           if (!mbar_wait(&sh.empty[s], ((it / STAGES) & 1) ^ 1)) { ok = false; break; }
           uint8_t *a_dst = ring + (size_t)s * STAGE_BYTES, *b_dst = a_dst + A_BYTES;
-          mbar_arrive_expect_tx(&sh.full[s], STAGE_BYTES);
+          const bool second = BN == 256 && bw > BN / 2;   // the second 128 rows of B are needed
+          mbar_arrive_expect_tx(&sh.full[s], second || BN != 256 ? STAGE_BYTES : STAGE_BYTES - B_BYTES / 2);
           tma_load_2d(a_dst, ma, &sh.full[s], ks * BK, tmi * BM);
           tma_load_2d(b_dst, mb, &sh.full[s], ks * BK, tni * BN);
-          if (BN == 256) tma_load_2d(b_dst + B_BYTES / 2, mb, &sh.full[s], ks * BK, tni * BN + BN / 2);
+          if (second) tma_load_2d(b_dst + B_BYTES / 2, mb, &sh.full[s], ks * BK, tni * BN + BN / 2);
         }
       }
       if (!ok) atomicExch(&sh.abort, 1);
@@ -306,6 +321,8 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
         if (!mbar_wait(&sh.acc_empty[a], ((tcount / NACC) & 1) ^ 1)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + a * BN;
+        // instruction descriptor with this tile's width in its N field
+        const uint32_t idesc = (Cfg::IDESC & ~(0x3Fu << 17)) | ((uint32_t)(tile_width<MODE, BN>(tni, ncols) >> 3) << 17);
         for (int ks = 0; ks < nslab; ++ks, ++it) {
           const int s = it % STAGES;
           if (!mbar_wait(&sh.full[s], (it / STAGES) & 1)) { ok = false; break; }
@@ -313,7 +330,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
           const uint32_t a_addr = smem_u32(ring + (size_t)s * STAGE_BYTES), b_addr = a_addr + A_BYTES;
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k)
-            umma_bf16(d_tmem, smem_desc(a_addr + k * 32), smem_desc(b_addr + k * 32), Cfg::IDESC, (ks | k) != 0);
+            umma_bf16(d_tmem, smem_desc(a_addr + k * 32), smem_desc(b_addr + k * 32), idesc, (ks | k) != 0);
           umma_commit(&sh.empty[s]);               // frees the slab once these MMAs have read it
         }
         if (ok) umma_commit(&sh.acc_full[a]);      // accumulator complete
