@@ -34,7 +34,7 @@ NCU_TRAFFIC: dict = {
     ("single_image", "merge"): 52310016 + 341248,
     ("single_image", "prepass"): 67227392 + 423936,
     ("single_image", "gram_density"): 3915520,
-    ("single_image", "assign"): 8372224,
+    ("single_image", "assign"): 8242176,
 }
 
 
