@@ -93,6 +93,7 @@ size_t carve_image(const pact_ctx *c, int N, char *base, ImgDesc *im) {
   cv.take(m.bstart, nblk * (size_t)m.bstride * sizeof(uint16_t));
   cv.take(m.csize, (size_t)Np * sizeof(int32_t));
   cv.take(m.cticket, (size_t)Np * sizeof(int32_t));
+  // chunk sums of the clusters that span several 16-member chunks: fewer than N / 8 rows
   cv.take(m.mpart, ((size_t)N / 8 + 2) * c->d * sizeof(float));
   return cv.off;
 }
