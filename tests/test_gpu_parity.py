@@ -84,6 +84,29 @@ def test_batch_of_sixteen_with_extreme_size_mix():
         assert not bad, f"N={img.N}: {bad}"
 
 
+def test_random_configurations():
+    """Forty seeded random combinations of size, shape, element type and parameters."""
+    rng = np.random.default_rng(2024)
+    for case in range(40):
+        N = int(rng.choice([rng.integers(1, 40), rng.integers(40, 400), rng.integers(400, 2600)]))
+        dtype = torch.bfloat16 if rng.random() < 0.7 else torch.float32
+        n_h, d_h = [(2, 32), (4, 128), (2, 64), (3, 16), (1, 64)][rng.integers(0, 5)]
+        kw = dict(seed=int(rng.integers(1, 10 ** 6)), N=N, T=int(rng.integers(0, 12)),
+                  n_blobs=int(max(1, min(60, N // int(rng.integers(3, 30)) + 1))),
+                  d=int(rng.choice([64, 256, 512, 1032])), n_h=n_h, d_h=d_h, dtype=dtype)
+        over = dict(lam=float(rng.choice([0.0, 0.1, 0.3, 0.5, 0.7, 0.9, 1.0, rng.random()])),
+                    d_c=float(rng.choice([0.0, 0.05, 0.2, 0.3, 0.5, 1.0, 2.0, rng.random()])),
+                    alpha=float(rng.choice([0.0, 1.0, 1.5, 3.0, rng.random() * 2])),
+                    d_n=float(rng.choice([0.5, 2.0, 4.0])))
+        out_dtype = torch.float32 if (dtype == torch.float32 or rng.random() < 0.5) else torch.bfloat16
+        wl = workloads.single_image(**kw)
+        outs, _ = gpu_reduce(wl, out_dtype, **over)
+        img = wl.images[0]
+        o = oracle_image(wl, img, **over)
+        bad = compare_image(o, outs[0], img, out_dtype == torch.bfloat16)
+        assert not bad, f"case {case} {kw} {over} {out_dtype}: {bad}; fragile: {fragile_report(o, over['d_c'], over['alpha'])}"
+
+
 # ------------------------------------------------------------------ edge and degenerate cases
 
 def _small(seed=21, N=700, T=9, **kw):
