@@ -82,7 +82,7 @@ __global__ void __launch_bounds__(kPreThreads, 2) k_prepass(const __grid_constan
   __shared__ double sm[kPreThreads * V];
   const T *Q = reinterpret_cast<const T *>(im.Q);
   const int c = t % cpp, gi = t / cpp;
-  constexpr int UQ = 8;
+  constexpr int UQ = 16;
   for (int cbase = 0; cbase < ncolv; cbase += cpp) {
     double acc[V];
 #pragma unroll
@@ -125,16 +125,22 @@ __global__ void __launch_bounds__(kPreThreads, 2) k_prepass(const __grid_constan
   __syncthreads();
   if (!last) return;
   __threadfence();
-  for (int col = t; col < bt.n_qcols; col += kPreThreads) {
-    double s = 0.0;
-    for (int h0 = 0; h0 < GQ; h0 += 16) {            // 16 partial sums in flight, added in index order
-      double v[16];
+  for (int col = t; col < bt.n_qcols; col += 2 * kPreThreads) {   // two columns per thread at a time
+    const int col2 = col + kPreThreads;
+    const bool two = col2 < bt.n_qcols;
+    double s = 0.0, s2 = 0.0;
+    for (int h0 = 0; h0 < GQ; h0 += 16) {            // 2 x 16 partial sums in flight, added in index order
+      double v[16], v2[16];
 #pragma unroll
-      for (int u = 0; u < 16; ++u) v[u] = h0 + u < GQ ? ld_cg_f64(&im.qpart[(size_t)(h0 + u) * bt.n_qcols + col]) : 0.0;
+      for (int u = 0; u < 16; ++u) {
+        v[u] = h0 + u < GQ ? ld_cg_f64(&im.qpart[(size_t)(h0 + u) * bt.n_qcols + col]) : 0.0;
+        v2[u] = (two && h0 + u < GQ) ? ld_cg_f64(&im.qpart[(size_t)(h0 + u) * bt.n_qcols + col2]) : 0.0;
+      }
 #pragma unroll
-      for (int u = 0; u < 16; ++u) s += v[u];
+      for (int u = 0; u < 16; ++u) { s += v[u]; s2 += v2[u]; }
     }
     im.qg[col] = s / (double)im.N;
+    if (two) im.qg[col2] = s2 / (double)im.N;
   }
   if (t == 0) im.cnt[16] = 0;
 }
