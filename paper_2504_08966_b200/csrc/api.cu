@@ -20,6 +20,7 @@ struct pact_ctx {
   int device;
   char err[256];
   long long launches;      // kernels launched by this context so far
+  int spin_limit;          // polls a bounded device wait makes before it raises PACT_ERR_TIMEOUT
   int prof_on;             // record an event after every stage of pact_reduce
   int prof_n;              // stages recorded by the last profiled call
   cudaEvent_t ev[kProfStages + 1];
@@ -87,14 +88,15 @@ size_t carve_image(const pact_ctx *c, int N, char *base, ImgDesc *im) {
   cv.take(m.cid, (size_t)Np * sizeof(int32_t));
   cv.take(m.best, (size_t)N * sizeof(unsigned long long));
   cv.take(m.label, (size_t)N * sizeof(int32_t));
-  const size_t nblk = ((size_t)N + 255) / 256;
-  m.bstride = Np + 8;
-  cv.take(m.blocklist, nblk * 256 * sizeof(int32_t));
-  cv.take(m.bstart, nblk * (size_t)m.bstride * sizeof(uint16_t));
+  const size_t nblk = ((size_t)N + kListBlock - 1) / kListBlock;
+  m.nbp = (int)rup(nblk, 8);
+  cv.take(m.blocklist, nblk * kListBlock * sizeof(int32_t));
+  cv.take(m.cnt_cb, (size_t)Np * m.nbp * sizeof(uint16_t));
+  cv.take(m.members, (size_t)N * sizeof(int4));
   cv.take(m.csize, (size_t)Np * sizeof(int32_t));
   cv.take(m.cticket, (size_t)Np * sizeof(int32_t));
-  // chunk sums of the clusters that span several 16-member chunks: fewer than N / 8 rows
-  cv.take(m.mpart, ((size_t)N / 8 + 2) * c->d * sizeof(float));
+  // two partial sums per CTA of k_merge (a range boundary cuts at most two clusters)
+  cv.take(m.mpart, (size_t)2 * merge_ctas(c->ccfg.sm_count, 1) * c->d * sizeof(float));
   return cv.off;
 }
 
@@ -171,7 +173,7 @@ pact_status check_image(const pact_ctx *c, const pact_image *g, bool need_euti, 
     if (!g->K_clu || !aligned16(g->K_clu) || !ld_ok(c, g->ldKc, c->d_k)) return PACT_ERR_INVALID_ARG;
   }
   if (need_out) {
-    if (g->N > merge_max_tokens(c->d, c->elt)) return PACT_ERR_UNSUPPORTED;
+    if (g->N > kMaxTokens) return PACT_ERR_UNSUPPORTED;
     if (!g->H || !aligned16(g->H) || !ld_ok(c, g->ldH, c->d) || !g->P) return PACT_ERR_INVALID_ARG;
     if (!g->H_out || !aligned16(g->H_out) || !g->P_out || !g->size_out || !g->counters)
       return PACT_ERR_INVALID_ARG;
@@ -252,6 +254,7 @@ pact_status pact_create(pact_ctx **out, int d, int n_qh, int n_kvh, int d_h, pac
     return PACT_ERR_CUDA;
   }
   c->umma = in == PACT_BF16 && umma_supported(c->d_k);
+  c->spin_limit = kSpinLimit;
   *out = c;
   return PACT_OK;
 }
@@ -378,7 +381,7 @@ pact_status pact_dbdpc(pact_ctx *ctx, const void *K, int64_t ldK, int N, const i
   launch_keynorm_gather(bt, N, bf, false, st);
   if (ctx->umma) CK(launch_gram_umma(bt, N, ctx->ccfg, st));
   else launch_gram(bt, N, bf, ctx->ccfg, st);
-  CK(launch_centers(bt, N, bf, ctx->ccfg, st));
+  CK(launch_centers(bt, N, bf, ctx->ccfg, ctx->spin_limit, st));
   if (ctx->umma) CK(launch_assign_umma(bt, N, true, ctx->ccfg, st));
   else launch_assign(bt, N, bf, ROWS_KEPT_LIST, ctx->ccfg, st);
   launch_label(bt, N, bf, ROWS_KEPT_LIST, st);
@@ -484,9 +487,10 @@ pact_status pact_merge(pact_ctx *ctx, const pact_image *img, const int32_t *labe
   CK(cudaMemsetAsync(m.cnt, 0, 32 * sizeof(int32_t), st));
   CK(cudaMemsetAsync(m.csize, 0, (size_t)m.Np * sizeof(int32_t), st));
   CK(cudaMemsetAsync(m.cticket, 0, (size_t)m.Np * sizeof(int32_t), st));
-  launch_lists(bt, img->N, ctx->in == PACT_BF16, false, st);
-  CK(launch_merge(bt, img->N, ctx->in == PACT_BF16, ctx->out == PACT_BF16, ctx->ccfg, st));
-  ctx->launches += 2;
+  CK(cudaMemsetAsync(m.cnt_cb, 0, (size_t)m.Np * m.nbp * sizeof(uint16_t), st));
+  CK(launch_lists(bt, img->N, ctx->in == PACT_BF16, false, ctx->spin_limit, st));
+  CK(launch_merge(bt, ctx->in == PACT_BF16, ctx->out == PACT_BF16, ctx->ccfg, st));
+  ctx->launches += lists_kernels(img->N, 1) + 1;
   CK(cudaGetLastError());
   CK(cudaMemcpyAsync(img->counters, m.cnt, sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
   return PACT_OK;
@@ -542,13 +546,13 @@ pact_status pact_reduce(pact_ctx *ctx, const pact_image *imgs, int B, const pact
     if (ctx->umma) CK(launch_gram_umma(bt, cmaxN, ctx->ccfg, st));
     else launch_gram(bt, cmaxN, bf, ctx->ccfg, st);
     CK(mark());
-    CK(launch_centers(bt, cmaxQ, bf, ctx->ccfg, st));  CK(mark());
+    CK(launch_centers(bt, cmaxQ, bf, ctx->ccfg, ctx->spin_limit, st));  CK(mark());
     if (ctx->umma) CK(launch_assign_umma(bt, cmaxN, false, ctx->ccfg, st));
     else launch_assign(bt, cmaxN, bf, ROWS_ALL, ctx->ccfg, st);
     CK(mark());
-    launch_lists(bt, cmaxN, bf, true, st);          CK(mark());
-    CK(launch_merge(bt, cmaxN, bf, ctx->out == PACT_BF16, ctx->ccfg, st));  CK(mark());
-    ctx->launches += 9;
+    CK(launch_lists(bt, cmaxN, bf, true, ctx->spin_limit, st));  CK(mark());
+    CK(launch_merge(bt, bf, ctx->out == PACT_BF16, ctx->ccfg, st));  CK(mark());
+    ctx->launches += 8 + lists_kernels(cmaxN, nb);
     CK(cudaGetLastError());
     for (int b = 0; b < nb; ++b)
       CK(cudaMemcpyAsync(bt.img[b].counters_user, bt.img[b].cnt, PACT_N_COUNTERS * sizeof(int32_t),

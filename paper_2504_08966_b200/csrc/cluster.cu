@@ -295,7 +295,7 @@ __global__ void k_spread_finish(const __grid_constant__ Batch bt, float *max_dis
 constexpr int kAdjRegs = 8;      // adjacency words per lane kept in registers: rows of up to 8192 survivors
 
 template <typename T>
-__global__ void __launch_bounds__(256) k_centers(const __grid_constant__ Batch bt, int keys_cap) {
+__global__ void __launch_bounds__(256) k_centers(const __grid_constant__ Batch bt, int keys_cap, int spin_limit) {
   using D = typename DistOf<T>::type;
   constexpr int V = Vec<T>::N;
   cooperative_groups::grid_group grid = cooperative_groups::this_grid();
@@ -367,7 +367,7 @@ __global__ void __launch_bounds__(256) k_centers(const __grid_constant__ Batch b
   // part 2: resolve
   int sweeps = 0, pending = 1;
   bool cached_done = false;
-  while (pending && sweeps < kSpinLimit) {
+  while (pending && sweeps < spin_limit) {
     pending = 0;
     ++sweeps;
     for (int r = gw; r < q; r += nwarps) {
@@ -650,7 +650,7 @@ void launch_gram(const Batch &bt, int maxN, bool bf16, const ClusterCfg &cfg, cu
   PACT_DISPATCH(bf16, k_gram_simt, <<<grid, 256, 0, st>>>(bt));
 }
 
-cudaError_t launch_centers(const Batch &bt, int maxQ, bool bf16, const ClusterCfg &cfg, cudaStream_t st) {
+cudaError_t launch_centers(const Batch &bt, int maxQ, bool bf16, const ClusterCfg &cfg, int spin_limit, cudaStream_t st) {
   // the densities of one image are staged in shared memory when they fit in a quarter of it; maxQ is
   // an estimate of the largest survivor count, an image with more reads them from global memory
   size_t smem = (size_t)maxQ * sizeof(unsigned long long);
@@ -664,7 +664,7 @@ cudaError_t launch_centers(const Batch &bt, int maxQ, bool bf16, const ClusterCf
   if (e != cudaSuccess) return e;
   if (per_sm < 1) return cudaErrorLaunchOutOfResources;
   if (per_sm > 4) per_sm = 4;
-  void *args[] = {(void *)&bt, (void *)&keys_cap};
+  void *args[] = {(void *)&bt, (void *)&keys_cap, (void *)&spin_limit};
   return cudaLaunchCooperativeKernel(fn, dim3(cfg.sm_count * per_sm), dim3(256), args, smem, st);
 }
 

@@ -13,7 +13,9 @@ constexpr int kRowsPerCta = 32;          // visual tokens handled by one CTA of 
 constexpr uint32_t kRhoShift = 30;       // density terms are summed as integers scaled by 2^30
 constexpr unsigned long long kBestInit = 0xFFFFFFFFFFFFFFFFull;
 constexpr int kCntSpread = 24;           // slot of cnt[]: largest key distance of a layer, as float bits
-constexpr int kSpinLimit = 1 << 20;      // passes a centre-selection warp makes before it gives up
+constexpr int kSpinLimit = 1 << 20;      // default number of polls a bounded device wait makes before it gives up
+constexpr int kListBlock = 256;          // tokens per block of the member-list sort
+constexpr int kMaxTokens = 1 << 18;      // most visual tokens per image
 
 // Per-image device pointers: the caller's buffers and the slices of the workspace.
 struct ImgDesc {
@@ -60,12 +62,13 @@ struct ImgDesc {
   int32_t *cid;          // [Np] cluster id of survivor r if it is a centre
   unsigned long long *best;  // [N] packed (distance bits << 32 | cluster id)
   int32_t *label;        // [N]
-  int32_t *blocklist;    // [ceil(N/256)][256] tokens of each block sorted by (cluster id, token)
-  uint16_t *bstart;      // [ceil(N/256)][bstride] tokens of the block with a cluster id below c
+  int32_t *blocklist;    // [ceil(N/256)][256] tokens of each block sorted by (cluster id, token); two-launch form of k_lists only
+  uint16_t *cnt_cb;      // [Np][nbp] members of cluster c in token block b; zero before k_lists
+  int4 *members;         // [N] {token, cluster, first member position of the cluster, cluster size}, cluster order
   int32_t *csize;        // [Np] members of cluster c
   int32_t *cticket;      // [Np] chunks of cluster c that are finished
-  float *mpart;          // [N/8 + 2][d] chunk sums
-  int32_t *cnt;          // [PACT_N_COUNTERS] + tickets: [16] global query, [19] member lists
+  float *mpart;          // [2 * merge CTAs][d] sums of the clusters that a range boundary of k_merge cuts
+  int32_t *cnt;          // [PACT_N_COUNTERS] + [16] ticket of the global query, [19] barrier of k_lists, [20] members of all clusters
   const int32_t *q_ptr;  // where the number of survivors lives (cnt[Q] or the caller's q_dev)
   const int32_t *m_ptr;  // where the number of pruned tokens lives
   const int32_t *C_ptr;  // where the number of clusters lives
@@ -74,7 +77,7 @@ struct ImgDesc {
   int32_t *center_idx_user, *C_user, *r_user;
   unsigned long long *tl; // timeline buffer of the instrumented build (PACT_TIMELINE), else unused
   int Np, Wp;            // padded survivor capacity and words per adjacency row
-  int bstride;           // entries per row of bstart
+  int nbp;               // entries per row of cnt_cb: token blocks, rounded up to a multiple of 8
 };
 
 struct Batch {
@@ -188,10 +191,32 @@ template <typename T> __device__ __forceinline__ void sumsq_accumulate(const uin
   }
 }
 
+// ---- L2 eviction hints -------------------------------------------------------------------------
+// The hidden states are read twice, by the scoring pass and by the merge, with everything else of the step
+// in between; together that is more than the L2 keeps under its default policy.  The first pass asks for
+// its lines to be evicted last, streams that are read once ask to be evicted first.
+__device__ __forceinline__ unsigned long long policy_evict_last() {
+  unsigned long long p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ unsigned long long policy_evict_first() {
+  unsigned long long p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint4 ldg_hint(const uint4 *p, unsigned long long policy) {
+  uint4 v;
+  asm volatile("ld.global.nc.L2::cache_hint.v4.u32 {%0, %1, %2, %3}, [%4], %5;"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p), "l"(policy));
+  return v;
+}
+
 // This lane's share (vectors lane, lane + 32, ... in ascending order) of the sum of squares of a
 // row of n elements, starting at vector `from`.  Up to U loads per lane are in flight at once.
-template <typename T, int U>
-__device__ __forceinline__ double row_sumsq_lane(const T *row, int n, int lane, int from = 0) {
+template <typename T, int U, bool HINT = false>
+__device__ __forceinline__ double row_sumsq_lane(const T *row, int n, int lane, int from = 0,
+                                                 unsigned long long policy = 0ull) {
   const int nv = n / Vec<T>::N;
   const uint4 *p = reinterpret_cast<const uint4 *>(row);
   double acc = 0.0;
@@ -199,7 +224,7 @@ __device__ __forceinline__ double row_sumsq_lane(const T *row, int n, int lane, 
     uint4 buf[U];
 #pragma unroll
     for (int u = 0; u < U; ++u)
-      if (v0 + 32 * u < nv) buf[u] = __ldg(p + v0 + 32 * u);
+      if (v0 + 32 * u < nv) buf[u] = HINT ? ldg_hint(p + v0 + 32 * u, policy) : __ldg(p + v0 + 32 * u);
 #pragma unroll
     for (int u = 0; u < U; ++u)
       if (v0 + 32 * u < nv) sumsq_accumulate<T>(buf[u], acc);

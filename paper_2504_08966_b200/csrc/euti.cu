@@ -57,7 +57,7 @@ __global__ void __launch_bounds__(kPreThreads, 2) k_prepass(const __grid_constan
       double nn = 1.0;
       if (!(im.flags & PACT_FLAG_NO_NORM)) {
         const T *hrow = reinterpret_cast<const T *>(im.H) + (size_t)(im.vis_start + tok) * im.ldH;
-        nn = sqrt(warp_sum(row_sumsq_lane<T, 16>(hrow, bt.d, lane)));
+        nn = sqrt(warp_sum(row_sumsq_lane<T, 16, true>(hrow, bt.d, lane, 0, policy_evict_last())));
       }
       if (lane == 0) im.nrm[tok] = nn;
     }
@@ -363,6 +363,9 @@ __global__ void __launch_bounds__(1024) k_select_gather(const __grid_constant__ 
     for (int r = gt; r < im.Np; r += gs) { im.rho_fix[r] = 0ull; im.csize[r] = 0; im.cticket[r] = 0; }
     for (int wd = gt; wd < im.Wp; wd += gs) { im.cmask[wd] = 0u; im.rmask[wd] = 0u; }
     for (int i = gt; i < N; i += gs) im.best[i] = kBestInit;
+    uint4 *tab = reinterpret_cast<uint4 *>(im.cnt_cb);
+    const int nq = im.Np * (im.nbp / 8);
+    for (int i = gt; i < nq; i += gs) tab[i] = make_uint4(0u, 0u, 0u, 0u);
   }
   if (t == 0) s_k = im.m_target;
   if (t < 256) hist[t] = 0;

@@ -31,7 +31,7 @@ void launch_center_key_gather(const Batch &bt, int maxN, bool bf16, cudaStream_t
 void launch_gram(const Batch &bt, int maxN, bool bf16, const ClusterCfg &cfg, cudaStream_t st);
 // density order, centre selection, cluster ids and centre keys in one cooperative kernel
 // maxQ: estimate of the largest number of survivors of an image (sizes the staging buffer only)
-cudaError_t launch_centers(const Batch &bt, int maxQ, bool bf16, const ClusterCfg &cfg, cudaStream_t st);
+cudaError_t launch_centers(const Batch &bt, int maxQ, bool bf16, const ClusterCfg &cfg, int spin_limit, cudaStream_t st);
 void launch_assign(const Batch &bt, int maxN, bool bf16, RowMode mode, const ClusterCfg &cfg, cudaStream_t st);
 void launch_label(const Batch &bt, int maxN, bool bf16, RowMode mode, cudaStream_t st);
 // layer choice: inverse norms of all keys of every layer, largest pair distance (any dtype), result
@@ -48,11 +48,12 @@ cudaError_t launch_assign_umma(const Batch &bt, int maxN, bool kept_rows, const 
 cudaError_t launch_spread_umma(const Batch &bt, int maxN, const ClusterCfg &cfg, cudaStream_t st);
 
 // merge.cu
-// member lists from label[] (from_best: labels are first formed from the nearest-centre pass, all tokens);
-// csize and cticket must be zero
-void launch_lists(const Batch &bt, int maxN, bool bf16, bool from_best, cudaStream_t st);
-cudaError_t launch_merge(const Batch &bt, int maxN, bool in_bf16, bool out_bf16, const ClusterCfg &cfg, cudaStream_t st);
+// member records in cluster order from label[] (from_best: labels are first formed from the nearest-centre
+// pass, all tokens); csize, cticket and cnt_cb must be zero.  spin_limit bounds the wait of its barrier.
+cudaError_t launch_lists(const Batch &bt, int maxN, bool bf16, bool from_best, int spin_limit, cudaStream_t st);
+int lists_kernels(int maxN, int B);        // kernels launch_lists launches (1, or 2 when the grid cannot be resident at once)
+cudaError_t launch_merge(const Batch &bt, bool in_bf16, bool out_bf16, const ClusterCfg &cfg, cudaStream_t st);
 cudaError_t merge_configure();
-int merge_max_tokens(int d, int elt);      // largest N the merge kernel takes (its chunk offsets live in shared memory)
+int merge_ctas(int sm_count, int B);       // CTAs per image of k_merge (sizes its scratch)
 
 }  // namespace pact

@@ -1,8 +1,19 @@
 // Merge (Eq. 10, Algorithm 3 step 4): one hidden state per cluster = mean of its members in
 // float accumulation and ascending token order; position id of the centre; cluster sizes;
 // text rows copied around the merged span.
+//
+//   k_lists  labels (reincorporation test of Eq. 8), then a stable counting sort of the tokens by
+//            cluster id: every block of 256 tokens sorts its own, an image-wide barrier, and every
+//            token writes one 16-byte record {token, cluster, first member position, cluster size}
+//            at its place in the cluster-sorted member array.  Also P', sizes and log sizes.
+//   k_merge  the member array (followed by the text rows) is cut into one contiguous range per CTA;
+//            a CTA streams the rows of its range with many loads in flight and no look-ups, keeps the
+//            running cluster in registers and writes a row out whenever the cluster id changes.
+//            Clusters cut by a range boundary leave partial sums; the last CTA to arrive adds them in
+//            range order, so the result does not depend on timing.
+#include <cooperative_groups.h>
+
 #include "kernels.cuh"
-#include "tma.cuh"
 
 namespace pact {
 
@@ -21,24 +32,13 @@ template <> __device__ __forceinline__ void store_vec8<__nv_bfloat16>(__nv_bfloa
   *reinterpret_cast<uint4 *>(p) = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
-// Loads 8 consecutive elements as float (one or two 16-byte loads).
-template <typename T> __device__ __forceinline__ void load8(const T *p, float (&x)[8]);
-template <> __device__ __forceinline__ void load8<__nv_bfloat16>(const __nv_bfloat16 *p, float (&x)[8]) {
-  load_vec<__nv_bfloat16>(p, x);
-}
-template <> __device__ __forceinline__ void load8<float>(const float *p, float (&x)[8]) {
-  float a[4], b[4];
-  load_vec<float>(p, a);
-  load_vec<float>(p + 4, b);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) { x[i] = a[i]; x[4 + i] = b[i]; }
-}
-
 // Eight consecutive elements of a row as loaded (not yet widened), so that many can be in flight.
 template <typename T> struct Raw8;
 template <> struct Raw8<__nv_bfloat16> {
   uint4 a;
-  __device__ __forceinline__ void load(const __nv_bfloat16 *p) { a = __ldg(reinterpret_cast<const uint4 *>(p)); }
+  __device__ __forceinline__ void load(const __nv_bfloat16 *p, unsigned long long pol) {
+    a = ldg_hint(reinterpret_cast<const uint4 *>(p), pol);
+  }
   __device__ __forceinline__ void add_to(float (&acc)[8]) const {
     float x[8];
     widen_vec<__nv_bfloat16>(a, x);
@@ -48,9 +48,9 @@ template <> struct Raw8<__nv_bfloat16> {
 };
 template <> struct Raw8<float> {
   uint4 a, b;
-  __device__ __forceinline__ void load(const float *p) {
-    a = __ldg(reinterpret_cast<const uint4 *>(p));
-    b = __ldg(reinterpret_cast<const uint4 *>(p) + 1);
+  __device__ __forceinline__ void load(const float *p, unsigned long long pol) {
+    a = ldg_hint(reinterpret_cast<const uint4 *>(p), pol);
+    b = ldg_hint(reinterpret_cast<const uint4 *>(p) + 1, pol);
   }
   __device__ __forceinline__ void add_to(float (&acc)[8]) const {
     float x[4], y[4];
@@ -61,14 +61,14 @@ template <> struct Raw8<float> {
   }
 };
 
-constexpr int kListBlock = 256;      // tokens per block of the member lists
-constexpr int kChunk = 16;           // members summed by one work item; the chunk-sum scratch of the workspace
-                                     // (N / 8 + 2 rows) is sized for this value: clusters of more than one chunk
-                                     // have at most 0.118 N chunks between them
-
 __device__ __forceinline__ int ld_cg_i32(const int *p) {
   int v;
   asm volatile("ld.global.cg.s32 %0, [%1];" : "=r"(v) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ int ld_acquire_i32(const int *p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
 __device__ __forceinline__ float4 ld_cg_f4(const float *p) {
@@ -78,123 +78,160 @@ __device__ __forceinline__ float4 ld_cg_f4(const float *p) {
 }
 
 // ---- member lists --------------------------------------------------------------------------------
-// grid (ceil(maxN / 256), B), 256 threads.  Block b sorts its 256 tokens by (cluster id, token) into
-// blocklist[b] (discarded tokens last) and writes bstart[b][c] = number of its tokens with a cluster id
-// below c, for c = 0..C.  The members of cluster c are then, in ascending token order, the entries
-// [bstart[b][c], bstart[b][c+1]) of blocklist[b] for b = 0, 1, ...  Cluster sizes are added up with
-// integer atomics.
+// grid (ceil(maxN / 256), B), 256 threads.
+// Part 1: block b sorts its 256 tokens by (cluster id, token), discarded tokens last; the first token of
+//   every run writes the run length to cnt_cb[c][b] (a table that is zero before the kernel) and adds it
+//   to csize[c].
+// Part 2 (after every block of the image has finished part 1): the member in sorted position t of block b
+//   belongs at  member_off[c] + (members of c in the blocks before b) + (its place in the run),  where
+//   member_off is the exclusive prefix sum of csize.  It writes its record there; the first member of a
+//   cluster also writes P', the size and its logarithm for the cluster's output row.
+// mode 0: both parts, separated by a barrier over the blocks of the image (all blocks must be resident:
+//         cooperative launch); mode 1: part 1 only, the sorted blocks go to blocklist; mode 2: part 2 only.
 // FROM_BEST: the labels are first formed here from the nearest-centre pass (survivors: cluster id of the
 // nearest centre, a centre its own id; pruned tokens: that id iff the distance is strictly below
-// alpha * d_c, else -1) and written out; otherwise label[] is given.
+// alpha * d_c, else -1) and written out; otherwise label[] is given, and an id outside [-1, C) is
+// dropped like -1 and reported through the status word.
+constexpr int kScanTile = kListBlock * 8;   // cluster sizes scanned per step of part 2
+constexpr int kNoLabel = 0x7fffffff;
+
 template <typename T, bool FROM_BEST>
-__global__ void __launch_bounds__(kListBlock) k_lists(const __grid_constant__ Batch bt) {
+__global__ void __launch_bounds__(kListBlock) k_lists(const __grid_constant__ Batch bt, int mode, int spin_limit) {
   using D = typename DistOf<T>::type;
   const ImgDesc &im = bt.img[blockIdx.y];
   TL_SCOPE(im, 8);
   const int N = im.N;
   const int nblk = (N + kListBlock - 1) / kListBlock;
-  const int b = blockIdx.x, t = threadIdx.x;
+  const int b = blockIdx.x, t = threadIdx.x, lane = t & 31, w = t >> 5;
   if (b >= nblk) return;
-  __shared__ int slab[kListBlock], sorted_lab[kListBlock];
+  __shared__ int slab[kListBlock], s_lab[kListBlock], s_tok[kListBlock];
+  __shared__ int excl[kScanTile];
+  __shared__ int wsum[kListBlock / 32];
+  __shared__ int s_carry;
+  const int C = min(*im.C_ptr, im.Np);
   const int i = b * kListBlock + t;
-  int lab = -1;
-  if (FROM_BEST) {
-    int joined = 0, dropped = 0, band = 0;
-    if (i < N) {
-      const int r = im.slot[i];                     // >= 0: survivor position; < 0: pruned
-      const unsigned long long pk = im.best[i];
-      lab = (int)(pk & 0xFFFFFFFFull);
-      const float dd = __uint_as_float((uint32_t)(pk >> 32));
-      if (r >= 0) {
-        if ((im.cmask[r >> 5] >> (r & 31)) & 1u) lab = im.cid[r];
-      } else {
-        if (D::in_band_t(dd, im)) ++band;
-        if (D::below_t(dd, im)) ++joined; else { lab = -1; ++dropped; }
+
+  if (mode != 2) {
+    int lab = -1;
+    if (FROM_BEST) {
+      int joined = 0, dropped = 0, band = 0;
+      if (i < N) {
+        const int r = im.slot[i];                     // >= 0: survivor position; < 0: pruned
+        const unsigned long long pk = im.best[i];
+        lab = (int)(pk & 0xFFFFFFFFull);
+        const float dd = __uint_as_float((uint32_t)(pk >> 32));
+        if (r >= 0) {
+          if ((im.cmask[r >> 5] >> (r & 31)) & 1u) lab = im.cid[r];
+        } else {
+          if (D::in_band_t(dd, im)) ++band;
+          if (D::below_t(dd, im)) ++joined; else { lab = -1; ++dropped; }
+        }
+        if (lab >= C) lab = -1;                       // only after a failed earlier stage
+        im.label[i] = lab;
+        if (im.label_user) im.label_user[i] = lab;
       }
-      im.label[i] = lab;
-      if (im.label_user) im.label_user[i] = lab;
-    }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      joined += __shfl_xor_sync(0xffffffffu, joined, o);
-      dropped += __shfl_xor_sync(0xffffffffu, dropped, o);
-      band += __shfl_xor_sync(0xffffffffu, band, o);
+      for (int o = 16; o > 0; o >>= 1) {
+        joined += __shfl_xor_sync(0xffffffffu, joined, o);
+        dropped += __shfl_xor_sync(0xffffffffu, dropped, o);
+        band += __shfl_xor_sync(0xffffffffu, band, o);
+      }
+      if (lane == 0) {
+        if (joined) atomicAdd(&im.cnt[PACT_CNT_R], joined);
+        if (dropped) atomicAdd(&im.cnt[PACT_CNT_DISCARDED], dropped);
+        if (band) atomicAdd(&im.cnt[PACT_CNT_BAND_ADC], band);
+      }
+    } else {
+      lab = i < N ? im.label[i] : -1;
+      if (lab >= C || lab < -1) {                     // a label the caller should not have passed
+        lab = -1;
+        atomicMin(&im.cnt[PACT_CNT_STATUS], (int)PACT_ERR_INVALID_ARG);
+      }
     }
-    if ((t & 31) == 0) {
-      if (joined) atomicAdd(&im.cnt[PACT_CNT_R], joined);
-      if (dropped) atomicAdd(&im.cnt[PACT_CNT_DISCARDED], dropped);
-      if (band) atomicAdd(&im.cnt[PACT_CNT_BAND_ADC], band);
-    }
-  } else {
-    lab = i < N ? im.label[i] : -1;
-  }
-  const int C = *im.C_ptr;
-  const int key = lab < 0 ? 0x7fffffff : lab;
-  slab[t] = key;
-  __syncthreads();
-  int rank = 0;
+    const int key = lab < 0 ? kNoLabel : lab;
+    slab[t] = key;
+    __syncthreads();
+    int rank = 0;
 #pragma unroll 8
-  for (int u = 0; u < kListBlock; ++u) {
-    const int o = slab[u];
-    rank += (o < key) || (o == key && u < t);
+    for (int u = 0; u < kListBlock; ++u) {
+      const int o = slab[u];
+      rank += (o < key) || (o == key && u < t);
+    }
+    s_lab[rank] = key;
+    s_tok[rank] = i;
+    __syncthreads();
+    if (mode == 1) im.blocklist[(size_t)b * kListBlock + t] = s_tok[t];
+  } else {
+    const int tok = im.blocklist[(size_t)b * kListBlock + t];
+    const int lab = tok < N ? im.label[tok] : -1;
+    s_tok[t] = tok;
+    s_lab[t] = (lab < 0 || lab >= C) ? kNoLabel : lab;
+    __syncthreads();
   }
-  sorted_lab[rank] = key;
-  im.blocklist[(size_t)b * kListBlock + rank] = i;
-  __syncthreads();
   // first position whose cluster id is >= c
   auto lower = [&](int c) {
     int lo = 0, hi = kListBlock;
     while (lo < hi) {
       const int mid = (lo + hi) >> 1;
-      if (sorted_lab[mid] < c) lo = mid + 1; else hi = mid;
+      if (s_lab[mid] < c) lo = mid + 1; else hi = mid;
     }
     return lo;
   };
-  uint16_t *row = im.bstart + (size_t)b * im.bstride;
-  for (int c = t; c <= C; c += kListBlock) row[c] = (uint16_t)lower(c);
-  {
-    const int c = sorted_lab[t];
-    if (c != 0x7fffffff && (t == 0 || sorted_lab[t - 1] != c)) atomicAdd(&im.csize[c], lower(c + 1) - t);
+  const int c = s_lab[t];
+  const bool valid = c != kNoLabel;
+  const int run0 = valid ? lower(c) : t;
+  if (mode != 2 && valid && run0 == t) {
+    const int len = lower(c + 1) - t;
+    im.cnt_cb[(size_t)c * im.nbp + b] = (uint16_t)len;
+    atomicAdd(&im.csize[c], len);
   }
-}
+  if (mode == 1) return;
+  TL_POINT(im, 13);
+  if (mode == 0) {
+    // every block of the image has published its run lengths before anyone reads them
+    __threadfence();
+    __syncthreads();
+    if (t == 0) {
+      atomicAdd(&im.cnt[19], 1);
+      int spins = 0;
+      while (ld_acquire_i32(&im.cnt[19]) < nblk) {
+        if (++spins > spin_limit) { atomicMin(&im.cnt[PACT_CNT_STATUS], (int)PACT_ERR_TIMEOUT); break; }
+        __nanosleep(40);
+      }
+    }
+    __syncthreads();
+    __threadfence();
+  }
+  TL_POINT(im, 14);
 
-// ---- Eq. 10 ------------------------------------------------------------------------------------------
-// Grid (X, B) with three CTAs of 256 threads per SM.  Work units are the chunks (kChunk members of one
-// cluster, ascending token order) followed by the text rows; CTA x takes units x, x + X, ...  For a unit
-// the CTA looks up the members (thread = block of the member lists), then every thread adds its columns
-// of the member rows in float with kMrgRows rows in flight, divides and stores.  A cluster of one chunk
-// is finished on the spot; otherwise the chunk sums go to scratch and the CTA that finishes the cluster's
-// last chunk adds them in chunk order.  Plain 16-byte loads: many small CTAs keep enough of them in
-// flight, and a CTA that waits on its look-up loads does not hold back the others.
-constexpr int kMrgThreads = 256;
-constexpr int kMrgRows = 4;                        // member rows in flight per thread
-constexpr int kMrgVpl = kMergeMaxD / 8 / kMrgThreads;   // 8-column groups per thread at the widest d
-
-template <typename T, typename O, int VPL>
-__global__ void __launch_bounds__(kMrgThreads, (VPL <= 2 && sizeof(T) == 2) ? 3 : 1)
-k_merge(const __grid_constant__ Batch bt) {
-  const ImgDesc &im = bt.img[blockIdx.y];
-  TL_SCOPE(im, 9);
-  const int t = threadIdx.x, lane = t & 31, w = t >> 5;
-  extern __shared__ int chunk_off[];               // [C + 1] first chunk of cluster c
-  __shared__ int wsum[kMrgThreads / 32];
-  __shared__ int s_carry, s_last;
-  __shared__ int members2[2][kChunk];              // member lists of the current and the previous unit
-  const int C = *im.C_ptr;
-  const int n_text = im.n_total - im.N;
-  const int d = bt.d, ng = d / 8;
-  const bool center_only = (im.flags & PACT_FLAG_CENTER_ONLY) != 0;
-  const T *H = reinterpret_cast<const T *>(im.H);
-  O *Ho = reinterpret_cast<O *>(im.H_out);
-  if (blockIdx.x == 0 && t == 0) im.cnt[PACT_CNT_N_OUT] = n_text + C;
+  // part 2
+  int before = 0, size = 0;                          // members of c in earlier blocks; members of c
+  if (valid) {
+    const uint4 *row = reinterpret_cast<const uint4 *>(im.cnt_cb + (size_t)c * im.nbp);
+    for (int v = 0; v * 8 < b; ++v) {
+      const uint4 x = __ldcg(row + v);
+      const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int cntk = (int)((xs[k >> 1] >> ((k & 1) * 16)) & 0xFFFFu);
+        if (v * 8 + k < b) before += cntk;
+      }
+    }
+    size = ld_cg_i32(&im.csize[c]);
+  }
+  // member_off[c] = cluster sizes below c, scanned kScanTile at a time
   if (t == 0) s_carry = 0;
   __syncthreads();
-  // chunk offsets: exclusive prefix sum of the chunks per cluster
-  for (int base = 0; base < C; base += kMrgThreads) {
-    const int c = base + t;
-    int nch = 0;
-    if (c < C) nch = center_only ? 1 : (im.csize[c] + kChunk - 1) / kChunk;
-    int x = nch;
+  int moff = 0;
+  for (int base = 0; base < C; base += kScanTile) {
+    int v8[8], s = 0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const int cc = base + t * 8 + k;
+      v8[k] = cc < C ? ld_cg_i32(&im.csize[cc]) : 0;
+      s += v8[k];
+    }
+    int x = s;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const int y = __shfl_up_sync(0xffffffffu, x, o);
@@ -204,247 +241,295 @@ k_merge(const __grid_constant__ Batch bt) {
     __syncthreads();
     int off = s_carry;
     for (int k = 0; k < w; ++k) off += wsum[k];
-    if (c < C) chunk_off[c] = off + x - nch;
+    int run = off + x - s;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { excl[t * 8 + k] = run; run += v8[k]; }
     __syncthreads();
-    if (t == kMrgThreads - 1) s_carry = off + x;
+    if (valid && c >= base && c < base + kScanTile) moff = excl[c - base];
+    if (t == kListBlock - 1) s_carry = run;
     __syncthreads();
   }
-  const int n_chunks = s_carry;
-  if (t == 0) chunk_off[C] = n_chunks;
-  __syncthreads();
-  TL_POINT(im, 13);
-  const int n_units = n_chunks + n_text;
-  const int nblk = (im.N + kListBlock - 1) / kListBlock;
+  if (b == 0 && t == 0) im.cnt[20] = s_carry;        // members in all clusters
+  if (!valid) return;
+  int pos = moff + before + (t - run0);
+  pos = max(0, min(pos, N - 1));                     // in bounds whatever an aborted stage left behind
+  const int tok = s_tok[t];
+  im.members[pos] = make_int4(tok, c, moff, size);
+  if (before == 0 && t == run0) {                    // first member of the cluster: the row's bookkeeping
+    const int dst = im.vis_start + c;
+    if (im.P_out) im.P_out[dst] = im.P[im.vis_start + min(max(im.cidx_ptr[c], 0), N - 1)];
+    if (im.size_out) im.size_out[dst] = size;
+    if (im.logw_out) im.logw_out[dst] = logf((float)size);   // Eq. 11: log of the token weight
+  }
+}
 
-  // units are handed out first come, first served (the order does not change any result)
-  // The member list and the next unit's number alternate between two slots: a thread can be at most one
-  // barrier behind, so the slots of unit n are rewritten (for unit n + 2) only after every thread has
-  // passed the barrier of unit n + 1, i.e. is done with unit n.  One CTA-wide barrier per unit.
-  __shared__ int s_next2[2];
-  int u = blockIdx.x, par = 0;
-  while (u < n_units) {
-    int c = -1, k = 0, nch = 1, size = 1, nm = 1, dst, ptok;
-    int *members = members2[par];
-    if (t == 0) s_next2[par] = gridDim.x + atomicAdd(&im.cnt[21], 1);   // needed only after this unit's rows
-    if (u >= n_chunks) {                           // a text row
-      const int tr = u - n_chunks;
-      const int src = tr < im.vis_start ? tr : tr + im.N;
-      dst = tr < im.vis_start ? tr : tr + C;
-      ptok = src;
-      if (t == 0) members[0] = src - im.vis_start; // relative to the visual span
-    } else {
-      int lo = 0, hi = C - 1;                      // last c with chunk_off[c] <= u
-      while (lo < hi) {
-        const int mid = (lo + hi + 1) >> 1;
-        if (chunk_off[mid] <= u) lo = mid; else hi = mid - 1;
-      }
-      c = lo;
-      k = u - chunk_off[c];
-      nch = chunk_off[c + 1] - chunk_off[c];
-      size = im.csize[c];
-      const int ctok = im.cidx_ptr[c];
-      dst = im.vis_start + c;
-      ptok = im.vis_start + ctok;
-      if (center_only) {
-        if (t == 0) members[0] = ctok;
-      } else {
-        const int m0 = k * kChunk, m1 = min(size, m0 + kChunk);
-        nm = m1 - m0;
-        int carry = 0;
-        if (nblk <= 32) {                           // one warp covers all blocks: no CTA-wide scan
-          if (w == 0) {
-            int s0 = 0, cntb = 0;
-            if (lane < nblk) {
-              const uint16_t *row = im.bstart + (size_t)lane * im.bstride;
-              s0 = row[c];
-              cntb = (int)row[c + 1] - s0;
-            }
-            int x = cntb;
+// ---- Eq. 10 ------------------------------------------------------------------------------------------
+// Grid (X, B), kMrgThreads threads, one CTA per SM.  Work items are the member records in cluster order
+// followed by the text rows; CTA x takes items [x per, (x + 1) per).  A thread owns VPL groups of 8 columns
+// and adds the rows of the running cluster in float; the loads of the next R rows are issued before the
+// current R rows are added.  A cluster that lies inside the range is divided and stored when the next one
+// begins.  A range boundary cuts at most two clusters per CTA: the one that began before the range (its
+// sum is set aside when it ends) and the one that goes on after it.  Their sums go to scratch (slot 0 and
+// slot 1 of the CTA) with a ticket each; the CTA that draws a cluster's last ticket adds the sums in range
+// order and stores the row, so the result does not depend on which CTA that is.
+constexpr int kMrgThreads = 512;
+constexpr int kMrgTile = 64;                        // records staged in shared memory at a time
+
+template <typename T, typename O, int VPL, int R>
+__global__ void __launch_bounds__(kMrgThreads, 1) k_merge(const __grid_constant__ Batch bt) {
+  const ImgDesc &im = bt.img[blockIdx.y];
+  TL_SCOPE(im, 9);
+  const int t = threadIdx.x;
+  __shared__ int4 s_rec[kMrgTile];                  // {row of H, cluster, first member position, size}
+  __shared__ int s_dst[kMrgTile];                   // output row
+  __shared__ float s_inv[kMrgTile];                 // 1 / size (1 for text rows and centre-only merging)
+  __shared__ int s_last;
+  const int C = min(*im.C_ptr, im.Np);
+  const int n_text = im.n_total - im.N;
+  const int d = bt.d, ng = d / 8;
+  const bool center_only = (im.flags & PACT_FLAG_CENTER_ONLY) != 0;
+  const T *H = reinterpret_cast<const T *>(im.H);
+  O *Ho = reinterpret_cast<O *>(im.H_out);
+  const int n_mem = center_only ? C : min(max(ld_cg_i32(&im.cnt[20]), 0), im.N);
+  const int total = n_mem + n_text;
+  const int X = gridDim.x, x = blockIdx.x;
+  const int per = (total + X - 1) / X;
+  const int lo = min(total, x * per), hi = min(total, lo + per);
+  if (x == 0 && t == 0) im.cnt[PACT_CNT_N_OUT] = n_text + C;
+  const unsigned long long pol_last_use = policy_evict_first();   // the rows are not read again
+
+  float acc[VPL][8], head[VPL][8];
+  int cur_c = -1, cur_off = 0, cur_size = 0, cur_dst = 0;
+  float cur_inv = 1.f;
+  int head_c = -1, head_off = 0, head_size = 0, head_dst = 0;   // the cluster that began before this range
+  float head_inv = 1.f;
+  bool head_open = false;                           // the running cluster is that one
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-              const int y = __shfl_up_sync(0xffffffffu, x, o);
-              if (lane >= o) x += y;
-            }
-            const int off = x - cntb;               // list position of this block's first member
-            const int a0 = max(off, m0), a1 = min(off + cntb, m1);
-            for (int m = a0; m < a1; ++m) members[m - m0] = im.blocklist[(size_t)lane * kListBlock + s0 + (m - off)];
-          }
-        } else
-        for (int bb0 = 0; bb0 < nblk; bb0 += kMrgThreads) {   // thread = block of the member lists
-          const int bb = bb0 + t;
-          int s0 = 0, cntb = 0;
-          if (bb < nblk) {                         // does not wait for the cluster size
-            const uint16_t *row = im.bstart + (size_t)bb * im.bstride;
-            s0 = row[c];
-            cntb = (int)row[c + 1] - s0;
-          }
-          int x = cntb;
+  for (int v = 0; v < VPL; ++v)
 #pragma unroll
-          for (int o = 1; o < 32; o <<= 1) {
-            const int y = __shfl_up_sync(0xffffffffu, x, o);
-            if (lane >= o) x += y;
-          }
-          if (bb0 > 0) __syncthreads();            // wsum of the previous round is consumed
-          if (lane == 31) wsum[w] = x;
-          __syncthreads();
-          int off = carry, tot = 0;
-#pragma unroll
-          for (int q = 0; q < kMrgThreads / 32; ++q) { if (q < w) off += wsum[q]; tot += wsum[q]; }
-          off += x - cntb;                         // list position of this block's first member
-          const int a0 = max(off, m0), a1 = min(off + cntb, m1);
-          for (int m = a0; m < a1; ++m) members[m - m0] = im.blocklist[(size_t)bb * kListBlock + s0 + (m - off)];
-          carry += tot;
-          if (carry >= m1) break;                  // uniform
-        }
-      }
-    }
-    __syncthreads();
-    float acc[VPL][8];
-#pragma unroll
-    for (int v = 0; v < VPL; ++v)
-#pragma unroll
-      for (int e = 0; e < 8; ++e) acc[v][e] = 0.f;
-#pragma unroll 1
-    for (int mi = 0; mi < nm; mi += kMrgRows) {
-      Raw8<T> x[kMrgRows][VPL];
-#pragma unroll
-      for (int r = 0; r < kMrgRows; ++r) {
-        if (mi + r < nm) {
-          const T *row = H + (size_t)(im.vis_start + members[mi + r]) * im.ldH;
-#pragma unroll
-          for (int v = 0; v < VPL; ++v) {
-            const int g = t + v * kMrgThreads;
-            if (g < ng) x[r][v].load(row + g * 8);
-          }
-        }
-      }
-#pragma unroll
-      for (int r = 0; r < kMrgRows; ++r) {
-        if (mi + r < nm) {
-#pragma unroll
-          for (int v = 0; v < VPL; ++v) {
-            const int g = t + v * kMrgThreads;
-            if (g < ng) x[r][v].add_to(acc[v]);
-          }
-        }
-      }
-    }
-    const float inv = center_only ? 1.0f : 1.0f / (float)size;   // one division per unit, not one per element
-    if (nch > 1) {
-      // scratch rows: the clusters that are summed in several chunks take theirs in cluster order
-      int base = 0;
-      for (int cc = lane; cc < c; cc += 32) {
-        const int n = chunk_off[cc + 1] - chunk_off[cc];
-        base += n > 1 ? n : 0;
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) base += __shfl_xor_sync(0xffffffffu, base, o);
-      float *part = im.mpart + (size_t)(base + k) * d;
-#pragma unroll
-      for (int v = 0; v < VPL; ++v) {
-        const int g = t + v * kMrgThreads;
-        if (g < ng) {
-          reinterpret_cast<float4 *>(part + g * 8)[0] = make_float4(acc[v][0], acc[v][1], acc[v][2], acc[v][3]);
-          reinterpret_cast<float4 *>(part + g * 8)[1] = make_float4(acc[v][4], acc[v][5], acc[v][6], acc[v][7]);
-        }
-      }
-      __threadfence();
-      __syncthreads();
-      if (t == 0) s_last = (atomicAdd(&im.cticket[c], 1) == nch - 1);
-      __syncthreads();
-      if (!s_last) { u = s_next2[par]; par ^= 1; continue; }
-      __threadfence();
-      const float *p0 = im.mpart + (size_t)base * d;
-#pragma unroll
-      for (int v = 0; v < VPL; ++v) {
-        const int g = t + v * kMrgThreads;
-        if (g < ng) {
-#pragma unroll
-          for (int e = 0; e < 8; ++e) acc[v][e] = 0.f;
-          for (int kk = 0; kk < nch; ++kk) {
-            const float4 a = ld_cg_f4(p0 + (size_t)kk * d + g * 8), bq = ld_cg_f4(p0 + (size_t)kk * d + g * 8 + 4);
-            acc[v][0] += a.x; acc[v][1] += a.y; acc[v][2] += a.z; acc[v][3] += a.w;
-            acc[v][4] += bq.x; acc[v][5] += bq.y; acc[v][6] += bq.z; acc[v][7] += bq.w;
-          }
-        }
-      }
-      if (t == 0) im.cticket[c] = 0;
-    }
+    for (int e = 0; e < 8; ++e) { acc[v][e] = 0.f; head[v][e] = 0.f; }
+
+  auto store_row = [&](const float (&a)[VPL][8], float inv, int dst) {
 #pragma unroll
     for (int v = 0; v < VPL; ++v) {
       const int g = t + v * kMrgThreads;
       if (g < ng) {
         float y[8];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) y[e] = acc[v][e] * inv;
+        for (int e = 0; e < 8; ++e) y[e] = a[v][e] * inv;
         store_vec8<O>(Ho + (size_t)dst * im.ldHo + g * 8, y);
       }
     }
-    if (t == 0) {
-      im.P_out[dst] = im.P[ptok];
-      im.size_out[dst] = size;
-      if (im.logw_out) im.logw_out[dst] = logf((float)size);   // Eq. 11: log of the token weight
+  };
+  auto issue = [&](Raw8<T> (&xr)[R][VPL], int j0, int tn) {
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      if (j0 + r < tn) {
+        const T *row = H + (size_t)s_rec[j0 + r].x * im.ldH;
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) {
+          const int g = t + v * kMrgThreads;
+          if (g < ng) xr[r][v].load(row + g * 8, pol_last_use);
+        }
+      }
     }
-    u = s_next2[par];
-    par ^= 1;
+  };
+  auto consume = [&](const Raw8<T> (&xr)[R][VPL], int j0, int tn) {
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      if (j0 + r < tn) {
+        const int4 rec = s_rec[j0 + r];
+        if (rec.y != cur_c) {                        // the next cluster begins (the same for all threads)
+          if (cur_c >= 0) {
+            if (head_open) {
+#pragma unroll
+              for (int v = 0; v < VPL; ++v)
+#pragma unroll
+                for (int e = 0; e < 8; ++e) head[v][e] = acc[v][e];
+              head_c = cur_c; head_off = cur_off; head_size = cur_size; head_dst = cur_dst; head_inv = cur_inv;
+              head_open = false;
+            } else {
+              store_row(acc, cur_inv, cur_dst);
+            }
+          } else {
+            head_open = rec.z < lo;
+          }
+#pragma unroll
+          for (int v = 0; v < VPL; ++v)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[v][e] = 0.f;
+          cur_c = rec.y; cur_off = rec.z; cur_size = rec.w;
+          cur_dst = s_dst[j0 + r]; cur_inv = s_inv[j0 + r];
+        }
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) {
+          const int g = t + v * kMrgThreads;
+          if (g < ng) xr[r][v].add_to(acc[v]);
+        }
+      }
+    }
+  };
+  // a cluster cut by a range boundary: sum to scratch, ticket, and the last one adds the sums in range order
+  auto cut = [&](float (&a)[VPL][8], int c, int off, int size, float inv, int dst, int slot) {
+    float *part = im.mpart + ((size_t)x * 2 + slot) * d;
+#pragma unroll
+    for (int v = 0; v < VPL; ++v) {
+      const int g = t + v * kMrgThreads;
+      if (g < ng) {
+        reinterpret_cast<float4 *>(part + g * 8)[0] = make_float4(a[v][0], a[v][1], a[v][2], a[v][3]);
+        reinterpret_cast<float4 *>(part + g * 8)[1] = make_float4(a[v][4], a[v][5], a[v][6], a[v][7]);
+      }
+    }
+    const int x0 = off / per, x1 = (off + size - 1) / per;
+    __threadfence();
+    __syncthreads();
+    if (t == 0) s_last = (atomicAdd(&im.cticket[c], 1) == x1 - x0);
+    __syncthreads();
+    const bool last = s_last != 0;
+    __syncthreads();                                 // s_last may be rewritten by the second cut cluster
+    if (!last) return;
+    __threadfence();
+#pragma unroll
+    for (int v = 0; v < VPL; ++v)
+#pragma unroll
+      for (int e = 0; e < 8; ++e) a[v][e] = 0.f;
+    for (int xx = x0; xx <= x1; ++xx) {
+      const float *p = im.mpart + ((size_t)xx * 2 + (xx < x1 ? 1 : 0)) * d;
+#pragma unroll
+      for (int v = 0; v < VPL; ++v) {
+        const int g = t + v * kMrgThreads;
+        if (g < ng) {
+          const float4 u = ld_cg_f4(p + g * 8), w = ld_cg_f4(p + g * 8 + 4);
+          a[v][0] += u.x; a[v][1] += u.y; a[v][2] += u.z; a[v][3] += u.w;
+          a[v][4] += w.x; a[v][5] += w.y; a[v][6] += w.z; a[v][7] += w.w;
+        }
+      }
+    }
+    if (t == 0) im.cticket[c] = 0;
+    store_row(a, inv, dst);
+  };
+
+  for (int t0 = lo; t0 < hi; t0 += kMrgTile) {
+    const int tn = min(kMrgTile, hi - t0);
+    __syncthreads();                                 // the previous tile's records are no longer needed
+    if (t < tn) {
+      const int g = t0 + t;
+      int4 rec;
+      int dst;
+      float inv = 1.f;
+      if (g < n_mem) {
+        if (center_only) rec = make_int4(im.cidx_ptr[g], g, g, 1);
+        else rec = __ldcg(im.members + g);
+        // in bounds whatever an aborted earlier stage left in the records
+        rec.x = min(max(rec.x, 0), im.N - 1) + im.vis_start;     // row of H
+        rec.y = min(max(rec.y, 0), C - 1);
+        rec.z = min(max(rec.z, 0), g);
+        rec.w = min(max(rec.w, g - rec.z + 1), n_mem - rec.z);
+        dst = im.vis_start + rec.y;
+        if (!center_only) inv = 1.0f / (float)rec.w;
+      } else {                                       // a text row: a cluster of its own, numbered after the real ones
+        const int tr = g - n_mem;
+        const int src = tr < im.vis_start ? tr : tr + im.N;
+        dst = tr < im.vis_start ? tr : tr + C;
+        rec = make_int4(src, C + tr, g, 1);
+        im.P_out[dst] = im.P[src];
+        im.size_out[dst] = 1;
+        if (im.logw_out) im.logw_out[dst] = 0.f;
+      }
+      s_rec[t] = rec;
+      s_dst[t] = dst;
+      s_inv[t] = inv;
+    }
+    __syncthreads();
+    Raw8<T> xa[R][VPL], xb[R][VPL];
+    issue(xa, 0, tn);
+#pragma unroll 1
+    for (int j0 = 0; j0 < tn; j0 += 2 * R) {
+      if (j0 + R < tn) issue(xb, j0 + R, tn);
+      consume(xa, j0, tn);
+      if (j0 + 2 * R < tn) issue(xa, j0 + 2 * R, tn);
+      if (j0 + R < tn) consume(xb, j0 + R, tn);
+    }
   }
+  if (cur_c < 0) return;                             // an empty range
+  const bool goes_on = cur_off + cur_size > hi;
+  if (head_open) {                                   // one cluster covers the whole range
+    cut(acc, cur_c, cur_off, cur_size, cur_inv, cur_dst, goes_on ? 1 : 0);
+    return;
+  }
+  if (head_c >= 0) cut(head, head_c, head_off, head_size, head_inv, head_dst, 0);
+  if (goes_on) cut(acc, cur_c, cur_off, cur_size, cur_inv, cur_dst, 1);
+  else store_row(acc, cur_inv, cur_dst);
 }
 
-void launch_lists(const Batch &bt, int maxN, bool bf16, bool from_best, cudaStream_t st) {
+// ---- launchers -----------------------------------------------------------------------------------
+
+namespace {
+int g_lists_resident = 0;                            // CTAs of k_lists that fit on the device at once
+}
+
+template <typename T, bool FB>
+static cudaError_t launch_lists_t(const Batch &bt, int maxN, int spin_limit, cudaStream_t st) {
   const dim3 grid((maxN + kListBlock - 1) / kListBlock, bt.B);
-  if (from_best) {
-    if (bf16) k_lists<__nv_bfloat16, true><<<grid, kListBlock, 0, st>>>(bt);
-    else k_lists<float, true><<<grid, kListBlock, 0, st>>>(bt);
-  } else {
-    k_lists<float, false><<<grid, kListBlock, 0, st>>>(bt);
+  if ((long long)grid.x * grid.y <= g_lists_resident) {
+    int mode = 0;
+    void *args[] = {(void *)&bt, (void *)&mode, (void *)&spin_limit};
+    return cudaLaunchCooperativeKernel((const void *)k_lists<T, FB>, grid, dim3(kListBlock), args, 0, st);
   }
-}
-
-static size_t g_merge_smem_max = 48 * 1024;
-
-template <typename T, typename O>
-static cudaError_t launch_merge_t(const Batch &bt, int maxN, const ClusterCfg &cfg, cudaStream_t st) {
-  const size_t smem = ((size_t)maxN + 2) * sizeof(int);
-  if (smem > g_merge_smem_max) return cudaErrorInvalidConfiguration;
-  int X = 3 * cfg.sm_count / bt.B;
-  if (X < 1) X = 1;
-  dim3 grid(X, bt.B);
-  if (bt.d <= kMrgThreads * 2 * 8) k_merge<T, O, 2><<<grid, kMrgThreads, smem, st>>>(bt);
-  else k_merge<T, O, kMrgVpl><<<grid, kMrgThreads, smem, st>>>(bt);
+  k_lists<T, FB><<<grid, kListBlock, 0, st>>>(bt, 1, spin_limit);
+  k_lists<T, FB><<<grid, kListBlock, 0, st>>>(bt, 2, spin_limit);
   return cudaGetLastError();
 }
 
-template <typename T, typename O> static cudaError_t merge_attr(int v) {
-  cudaError_t e = cudaFuncSetAttribute(k_merge<T, O, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, v);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(k_merge<T, O, kMrgVpl>, cudaFuncAttributeMaxDynamicSharedMemorySize, v);
+cudaError_t launch_lists(const Batch &bt, int maxN, bool bf16, bool from_best, int spin_limit, cudaStream_t st) {
+  if (from_best) {
+    if (bf16) return launch_lists_t<__nv_bfloat16, true>(bt, maxN, spin_limit, st);
+    return launch_lists_t<float, true>(bt, maxN, spin_limit, st);
+  }
+  return launch_lists_t<float, false>(bt, maxN, spin_limit, st);
+}
+
+int lists_kernels(int maxN, int B) {
+  return (long long)((maxN + kListBlock - 1) / kListBlock) * B <= g_lists_resident ? 1 : 2;
+}
+
+int merge_ctas(int sm_count, int B) {
+  const int X = sm_count / B;
+  return X < 1 ? 1 : X;
+}
+
+template <typename T, typename O>
+static cudaError_t launch_merge_t(const Batch &bt, const ClusterCfg &cfg, cudaStream_t st) {
+  dim3 grid(merge_ctas(cfg.sm_count, bt.B), bt.B);
+  constexpr int R1 = sizeof(T) == 2 ? 8 : 4;         // rows per batch; two batches are in flight
+  if (bt.d <= kMrgThreads * 8) k_merge<T, O, 1, R1><<<grid, kMrgThreads, 0, st>>>(bt);
+  else k_merge<T, O, kMergeMaxD / 8 / kMrgThreads, R1 / 2><<<grid, kMrgThreads, 0, st>>>(bt);
+  return cudaGetLastError();
 }
 
 cudaError_t merge_configure() {
-  int dev = 0, optin = 0;
+  int dev = 0, sms = 0, per_sm = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
-  e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return e;
-  g_merge_smem_max = (size_t)optin - 2048;
-  const int v = (int)g_merge_smem_max;
-  e = merge_attr<__nv_bfloat16, __nv_bfloat16>(v);
-  if (e == cudaSuccess) e = merge_attr<__nv_bfloat16, float>(v);
-  if (e == cudaSuccess) e = merge_attr<float, __nv_bfloat16>(v);
-  if (e == cudaSuccess) e = merge_attr<float, float>(v);
-  return e;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_lists<__nv_bfloat16, true>, kListBlock, 0);
+  if (e != cudaSuccess) return e;
+  int m = per_sm;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_lists<float, true>, kListBlock, 0);
+  if (e != cudaSuccess) return e;
+  m = per_sm < m ? per_sm : m;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_lists<float, false>, kListBlock, 0);
+  if (e != cudaSuccess) return e;
+  m = per_sm < m ? per_sm : m;
+  g_lists_resident = m * sms;
+  return cudaSuccess;
 }
 
-// largest N the merge kernel takes: its chunk offsets live in shared memory
-int merge_max_tokens(int d, int elt) {
-  (void)d; (void)elt;
-  return (int)(g_merge_smem_max / sizeof(int)) - 2;
-}
-
-cudaError_t launch_merge(const Batch &bt, int maxN, bool in_bf16, bool out_bf16, const ClusterCfg &cfg, cudaStream_t st) {
-  if (in_bf16) return out_bf16 ? launch_merge_t<__nv_bfloat16, __nv_bfloat16>(bt, maxN, cfg, st)
-                               : launch_merge_t<__nv_bfloat16, float>(bt, maxN, cfg, st);
-  return out_bf16 ? launch_merge_t<float, __nv_bfloat16>(bt, maxN, cfg, st) : launch_merge_t<float, float>(bt, maxN, cfg, st);
+cudaError_t launch_merge(const Batch &bt, bool in_bf16, bool out_bf16, const ClusterCfg &cfg, cudaStream_t st) {
+  if (in_bf16) return out_bf16 ? launch_merge_t<__nv_bfloat16, __nv_bfloat16>(bt, cfg, st)
+                               : launch_merge_t<__nv_bfloat16, float>(bt, cfg, st);
+  return out_bf16 ? launch_merge_t<float, __nv_bfloat16>(bt, cfg, st) : launch_merge_t<float, float>(bt, cfg, st);
 }
 
 }  // namespace pact
