@@ -31,10 +31,6 @@ N_COPIES = 4          # input copies rotated between steps so that no step finds
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
 # (workload, kernel) -> bytes; absent = not captured for the kernel as it stands
 NCU_TRAFFIC: dict = {
-    ("single_image", "merge"): 52310016 + 341248,
-    ("single_image", "prepass"): 67236352 + 438272,
-    ("single_image", "gram_density"): 3915520,
-    ("single_image", "assign"): 8242176,
 }
 
 
@@ -439,9 +435,7 @@ def main():
     t_roof = max(t_hbm, t_tc) * B
     n_qcols = wl.n_qh * wl.d_h
     alg = {   # algorithmic bytes (hbm) or flops (tensor) of one launch of each kernel, image 0 scaled by B
-        "prepass": ("hbm", img0.N * d * 2.0 + img0.N * d_k * 2.0 + img0.N * n_qcols * 2.0),
-        "logits": ("hbm", img0.N * d_k * 2.0 + img0.N * wl.n_qh * 8.0),
-        "select_gather": ("hbm", 2.0 * q * d_k * 2.0 + img0.N * 4.0),
+        "euti": ("hbm", img0.N * d * 2.0 + img0.N * d_k * 2.0 + img0.N * n_qcols * 2.0 + q * d_k * 2.0),
         "gram_density": ("tensor", 2.0 * d_k * (q * (q + 1) / 2)),
         "assign": ("tensor", 2.0 * d_k * img0.N * Cn),
         "merge": ("hbm", (q + r) * d * 2.0 + Cn * d * 2.0 + 2 * T * d * 2.0),

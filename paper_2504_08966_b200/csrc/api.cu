@@ -9,7 +9,7 @@
 
 using namespace pact;
 
-constexpr int kProfStages = 9;
+constexpr int kProfStages = 6;
 
 struct pact_ctx {
   int d, n_qh, n_kvh, d_h, d_k, n_qcols;
@@ -32,9 +32,7 @@ struct pact_graph {
   int kernels;             // kernels one replay launches
 };
 
-static const char *const kStageNames[kProfStages] = {
-    "prepass", "logits", "scores", "select_gather", "gram_density", "centers", "assign", "label_lists",
-    "merge"};
+static const char *const kStageNames[kProfStages] = {"euti", "gram_density", "centers", "assign", "label_lists", "merge"};
 
 namespace {
 
@@ -55,16 +53,17 @@ size_t carve_image(const pact_ctx *c, int N, char *base, ImgDesc *im) {
   ImgDesc tmp;
   ImgDesc &m = im ? *im : tmp;
   Carver cv{base};
-  const int G = (N + kRowsPerCta - 1) / kRowsPerCta;
   const int Np = (int)rup((size_t)N, 128);
   const int Wp = Np / 32;
   m.Np = Np;
   m.Wp = Wp;
-  cv.take(m.cnt, 32 * sizeof(int32_t));
+  cv.take(m.cnt, (size_t)(kCntInts + kTickInts) * sizeof(int32_t));
+  if (m.cnt) m.tick = m.cnt + kCntInts;
   cv.take(m.qpart, (size_t)kQPartRows * c->n_qcols * sizeof(double));
   cv.take(m.qg, (size_t)c->n_qcols * sizeof(double));
   cv.take(m.E, (size_t)N * c->n_qh * sizeof(double));
-  cv.take(m.part, (size_t)G * c->n_qh * 2 * sizeof(double));
+  cv.take(m.part, (size_t)((N + kRowsPerCta - 1) / kRowsPerCta) * c->n_qh * 2 * sizeof(double));
+  cv.take(m.ghist, ((size_t)1 << kHistBits) * sizeof(int32_t));
   cv.take(m.nrm, (size_t)N * sizeof(double));
   cv.take(m.score, (size_t)N * sizeof(float));
   cv.take(m.keep, (size_t)N);
@@ -230,6 +229,7 @@ pact_status pact_create(pact_ctx **out, int d, int n_qh, int n_kvh, int d_h, pac
   const int v = in == PACT_BF16 ? 8 : 4;
   if (d % 8 != 0 || d_h % v != 0) return PACT_ERR_UNSUPPORTED;
   if (d > kMergeMaxD || n_qh > 256) return PACT_ERR_UNSUPPORTED;
+  if ((n_qh * d_h / v + 7) / 8 > kTickInts) return PACT_ERR_UNSUPPORTED;   // one ticket per 128-byte column group of Q
   pact_ctx *c = new (std::nothrow) pact_ctx;
   if (!c) return PACT_ERR_INVALID_ARG;
   memset(c, 0, sizeof(*c));
@@ -317,11 +317,9 @@ pact_status pact_importance(pact_ctx *ctx, const pact_image *img, const pact_par
   m.score_user = score;
   set_params(m, p, img->N);
   point_counts_at_workspace(m);
-  CK(cudaMemsetAsync(m.cnt, 0, 32 * sizeof(int32_t), st));
-  launch_prepass(bt, img->N, ctx->in == PACT_BF16, st);
-  launch_logits(bt, img->N, ctx->in == PACT_BF16, st);
-  launch_scores(bt, img->N, st);
-  ctx->launches += 3;
+  CK(cudaMemsetAsync(m.cnt, 0, (kCntInts + kTickInts) * sizeof(int32_t), st));
+  CK(launch_euti(bt, img->N, ctx->in == PACT_BF16, 1, st));
+  ctx->launches += euti_kernels(1);
   CK(cudaGetLastError());
   return PACT_OK;
 }
@@ -377,7 +375,7 @@ pact_status pact_dbdpc(pact_ctx *ctx, const void *K, int64_t ldK, int N, const i
   m.kept_idx = const_cast<int32_t *>(idx);
   m.q_ptr = q_dev;
   m.rho_user = rho; m.center_idx_user = center_idx; m.C_user = C_dev; m.label_user = label;
-  CK(cudaMemsetAsync(m.cnt, 0, 32 * sizeof(int32_t), st));
+  CK(cudaMemsetAsync(m.cnt, 0, (kCntInts + kTickInts) * sizeof(int32_t), st));
   launch_keynorm_gather(bt, N, bf, false, st);
   if (ctx->umma) CK(launch_gram_umma(bt, N, ctx->ccfg, st));
   else launch_gram(bt, N, bf, ctx->ccfg, st);
@@ -416,7 +414,7 @@ pact_status pact_key_spread(pact_ctx *ctx, const void *const *K_layers, int n_la
       carve_image(ctx, N, (char *)ws + (size_t)b * per_img, &m);
       m.N = N; m.Kc = K_layers[base + b]; m.ldKc = ldK;
       point_counts_at_workspace(m);
-      CK(cudaMemsetAsync(m.cnt, 0, 32 * sizeof(int32_t), st));
+      CK(cudaMemsetAsync(m.cnt, 0, (kCntInts + kTickInts) * sizeof(int32_t), st));
     }
     launch_key_rnorm(bt, N, bf, st);
     if (ctx->umma) CK(launch_spread_umma(bt, N, ctx->ccfg, st));
@@ -452,7 +450,7 @@ pact_status pact_reincorporate(pact_ctx *ctx, const void *K, int64_t ldK, int N,
   m.pruned_idx = const_cast<int32_t *>(pruned_idx);
   m.m_ptr = m_dev; m.C_ptr = C_dev; m.cidx_ptr = center_idx;
   m.label = label;                      // updated in place
-  CK(cudaMemsetAsync(m.cnt, 0, 32 * sizeof(int32_t), st));
+  CK(cudaMemsetAsync(m.cnt, 0, (kCntInts + kTickInts) * sizeof(int32_t), st));
   launch_center_key_gather(bt, N, bf, st);
   launch_assign(bt, N, bf, ROWS_PRUNED_LIST, ctx->ccfg, st);
   launch_label(bt, N, bf, ROWS_PRUNED_LIST, st);
@@ -484,7 +482,7 @@ pact_status pact_merge(pact_ctx *ctx, const pact_image *img, const int32_t *labe
   point_counts_at_workspace(m);
   m.label = const_cast<int32_t *>(label);
   m.C_ptr = C_dev; m.cidx_ptr = center_idx;
-  CK(cudaMemsetAsync(m.cnt, 0, 32 * sizeof(int32_t), st));
+  CK(cudaMemsetAsync(m.cnt, 0, (kCntInts + kTickInts) * sizeof(int32_t), st));
   CK(cudaMemsetAsync(m.csize, 0, (size_t)m.Np * sizeof(int32_t), st));
   CK(cudaMemsetAsync(m.cticket, 0, (size_t)m.Np * sizeof(int32_t), st));
   CK(cudaMemsetAsync(m.cnt_cb, 0, (size_t)m.Np * m.nbp * sizeof(uint16_t), st));
@@ -529,7 +527,7 @@ pact_status pact_reduce(pact_ctx *ctx, const pact_image *imgs, int B, const pact
       cmaxN = g->N > cmaxN ? g->N : cmaxN;
       const int qest = g->N - m.m_target + 64 < g->N ? g->N - m.m_target + 64 : g->N;   // survivors, with room for ties
       cmaxQ = qest > cmaxQ ? qest : cmaxQ;
-      CK(cudaMemsetAsync(m.cnt, 0, 32 * sizeof(int32_t), st));
+      CK(cudaMemsetAsync(m.cnt, 0, (kCntInts + kTickInts) * sizeof(int32_t), st));
     }
     int stage = 0;
     auto mark = [&]() -> cudaError_t {
@@ -539,10 +537,7 @@ pact_status pact_reduce(pact_ctx *ctx, const pact_image *imgs, int B, const pact
       return cudaEventRecord(ctx->ev[stage], st);
     };
     if (ctx->prof_on && b0 == 0) CK(cudaEventRecord(ctx->ev[0], st));
-    launch_prepass(bt, cmaxN, bf, st);              CK(mark());
-    launch_logits(bt, cmaxN, bf, st);               CK(mark());
-    launch_scores(bt, cmaxN, st);                   CK(mark());
-    launch_select_gather(bt, cmaxN, bf, true, st);  CK(mark());
+    CK(launch_euti(bt, cmaxN, bf, 0, st));  CK(mark());
     if (ctx->umma) CK(launch_gram_umma(bt, cmaxN, ctx->ccfg, st));
     else launch_gram(bt, cmaxN, bf, ctx->ccfg, st);
     CK(mark());
@@ -552,7 +547,7 @@ pact_status pact_reduce(pact_ctx *ctx, const pact_image *imgs, int B, const pact
     CK(mark());
     CK(launch_lists(bt, cmaxN, bf, true, ctx->spin_limit, st));  CK(mark());
     CK(launch_merge(bt, bf, ctx->out == PACT_BF16, ctx->ccfg, st));  CK(mark());
-    ctx->launches += 8 + lists_kernels(cmaxN, nb);
+    ctx->launches += euti_kernels(0) + 4 + lists_kernels(cmaxN, nb);
     CK(cudaGetLastError());
     for (int b = 0; b < nb; ++b)
       CK(cudaMemcpyAsync(bt.img[b].counters_user, bt.img[b].cnt, PACT_N_COUNTERS * sizeof(int32_t),

@@ -7,6 +7,10 @@
 #include <cooperative_groups.h>
 
 #include "kernels.cuh"
+#ifdef PACT_TL_EUTI
+#undef TL_POINT
+#define TL_POINT(im, kid)
+#endif
 
 namespace pact {
 

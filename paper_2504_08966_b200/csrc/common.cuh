@@ -16,6 +16,8 @@ constexpr int kCntSpread = 24;           // slot of cnt[]: largest key distance 
 constexpr int kSpinLimit = 1 << 20;      // default number of polls a bounded device wait makes before it gives up
 constexpr int kListBlock = 256;          // tokens per block of the member-list sort
 constexpr int kMaxTokens = 1 << 18;      // most visual tokens per image
+constexpr int kCntInts = 64;             // counters and tickets at the head of an image's workspace ...
+constexpr int kTickInts = 1024;          // ... followed by the tickets of k_qsum; both are cleared when a call starts
 
 // Per-image device pointers: the caller's buffers and the slices of the workspace.
 struct ImgDesc {
@@ -38,7 +40,8 @@ struct ImgDesc {
   double *qpart;         // [kQPartRows][n_qcols] partial column sums of Q
   double *qg;            // [n_qcols] global query
   double *E;             // [N][n_qh] exp(logit - CTA max)
-  double *part;          // [G][n_qh][2] per-CTA (max, sum)
+  double *part;          // [G][n_qh][2] per-CTA (max, sum) of k_tokens, G = ceil(N / 32)
+  int32_t *ghist;        // [2^kHistBits] scores per bin of their top key bits
   double *nrm;           // [N] hidden-state norms
   float *score;          // [N]
   unsigned char *keep;   // [N]
@@ -68,6 +71,7 @@ struct ImgDesc {
   int32_t *csize;        // [Np] members of cluster c
   int32_t *cticket;      // [Np] chunks of cluster c that are finished
   float *mpart;          // [2 * merge CTAs][d] sums of the clusters that a range boundary of k_merge cuts
+  int32_t *tick;         // [kTickInts] tickets of k_qsum, one per column group; zero when a call starts (cleared with cnt)
   int32_t *cnt;          // [PACT_N_COUNTERS] + [16] ticket of the global query, [19] barrier of k_lists, [20] members of all clusters
   const int32_t *q_ptr;  // where the number of survivors lives (cnt[Q] or the caller's q_dev)
   const int32_t *m_ptr;  // where the number of pruned tokens lives
@@ -191,6 +195,16 @@ template <typename T> __device__ __forceinline__ void sumsq_accumulate(const uin
   }
 }
 
+// ---- programmatic dependent launch ----------------------------------------------------------------------
+// The step is a chain of short kernels.  A kernel launched with the programmatic-serialization attribute may
+// start while its predecessor in the stream is still running: pdl_wait() blocks until the predecessor has
+// finished and its writes are visible; whatever does not depend on it (set-up, and in k_tokens the whole pass
+// over the hidden states) runs before.  pdl_trigger() in the predecessor lets the successor's CTAs be
+// scheduled from then on.  Every CTA of every kernel calls pdl_wait() before it returns, so completion of a
+// kernel implies completion of all kernels before it.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- L2 eviction hints -------------------------------------------------------------------------
 // The hidden states are read twice, by the scoring pass and by the merge, with everything else of the step
 // in between; together that is more than the L2 keeps under its default policy.  The first pass asks for
@@ -212,6 +226,25 @@ __device__ __forceinline__ uint4 ldg_hint(const uint4 *p, unsigned long long pol
   return v;
 }
 
+// The same with a compile-time byte offset folded into the instruction: a run of such loads from one base
+// needs one address register, not one per load.
+template <int OFF>
+__device__ __forceinline__ uint4 ldg_hint_off(const uint4 *p, unsigned long long policy) {
+  uint4 v;
+  asm volatile("ld.global.nc.L2::cache_hint.v4.u32 {%0, %1, %2, %3}, [%4 + %6], %5;"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p), "l"(policy), "n"(OFF));
+  return v;
+}
+
+// buf[u] = base[32 u] for the u with v0 + 32 u < nv, all from one address register
+template <int U, int I>
+__device__ __forceinline__ void load_run_hint(uint4 (&buf)[U], const uint4 *base, int v0, int nv, unsigned long long policy) {
+  if constexpr (I < U) {
+    if (v0 + 32 * I < nv) buf[I] = ldg_hint_off<32 * I * 16>(base, policy);
+    load_run_hint<U, I + 1>(buf, base, v0, nv, policy);
+  }
+}
+
 // This lane's share (vectors lane, lane + 32, ... in ascending order) of the sum of squares of a
 // row of n elements, starting at vector `from`.  Up to U loads per lane are in flight at once.
 template <typename T, int U, bool HINT = false>
@@ -222,12 +255,20 @@ __device__ __forceinline__ double row_sumsq_lane(const T *row, int n, int lane, 
   double acc = 0.0;
   for (int v0 = from + lane; v0 < nv; v0 += 32 * U) {
     uint4 buf[U];
+    if (HINT) {
+      load_run_hint<U, 0>(buf, p + v0, v0, nv, policy);
+    } else {
 #pragma unroll
-    for (int u = 0; u < U; ++u)
-      if (v0 + 32 * u < nv) buf[u] = HINT ? ldg_hint(p + v0 + 32 * u, policy) : __ldg(p + v0 + 32 * u);
+      for (int u = 0; u < U; ++u)
+        if (v0 + 32 * u < nv) buf[u] = __ldg(p + v0 + 32 * u);
+    }
 #pragma unroll
-    for (int u = 0; u < U; ++u)
+    for (int u = 0; u < U; ++u) {
       if (v0 + 32 * u < nv) sumsq_accumulate<T>(buf[u], acc);
+      // one vector after the other: left to itself the compiler widens all U vectors at once for the sake of
+      // instruction-level parallelism and spills the loaded data, which serialises the loads
+      if (u + 1 < U) asm volatile("" : "+r"(buf[u + 1].x), "+d"(acc));
+    }
   }
   return acc;
 }

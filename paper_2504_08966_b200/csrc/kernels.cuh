@@ -4,16 +4,37 @@
 
 namespace pact {
 
+// Launches a kernel; pdl: with the programmatic-serialization attribute (it may start before its predecessor in
+// the stream has finished and must call pdl_wait() before it reads what the predecessor wrote).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool pdl,
+                            Args &&...args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 constexpr int kMergeMaxD = 256 * 4 * 8;   // widest hidden state the merge kernel holds in registers
 
 // how a kernel finds its rows
 enum RowMode { ROWS_ALL = 0, ROWS_KEPT_LIST = 1, ROWS_PRUNED_LIST = 2 };
 
 // euti.cu
-constexpr int kQPartRows = 64;            // most partial sums of Q the prepass writes per image
-void launch_prepass(const Batch &bt, int maxN, bool bf16, cudaStream_t st);
-void launch_logits(const Batch &bt, int maxN, bool bf16, cudaStream_t st);
-void launch_scores(const Batch &bt, int maxN, cudaStream_t st);
+constexpr int kQPartRows = 32;            // most row blocks the column sums of Q are split into
+constexpr int kHistBits = 12;             // key bits of the first-level histogram of the threshold selection
+constexpr int kHistShift = 32 - kHistBits; // a key's bin in that histogram is key >> kHistShift
+// Algorithm 1.  mode 0: scores, threshold, lists, survivor keys (four kernels; the first also clears what later
+// kernels accumulate into); mode 1: scores only (three kernels).
+cudaError_t launch_euti(const Batch &bt, int maxN, bool bf16, int mode, cudaStream_t st);
+int euti_kernels(int mode);
 // threshold + ordered compaction; gather: also copy the survivor keys and clear the accumulators
 void launch_select_gather(const Batch &bt, int maxN, bool bf16, bool gather, cudaStream_t st);
 cudaError_t euti_configure(int n_qcols, int n_qh);
