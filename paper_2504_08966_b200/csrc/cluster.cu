@@ -286,34 +286,44 @@ __global__ void k_spread_finish(const __grid_constant__ Batch bt, float *max_dis
 // schedule that only takes final decisions reproduces it (the argument of Appendix D.2).  A row becomes
 //   removed  once an earlier neighbour is a centre,
 //   a centre once every earlier neighbour is removed.
-// Both facts are monotone bits, so rows are resolved asynchronously: each warp owns rows, re-reads
-// the two bit masks and decides what it can, until all its rows are decided.
+// Both facts are monotone bits, so rows are resolved asynchronously from two bit masks in global memory.
+// The masks are a few hundred bytes that every row depends on: thousands of warps polling them directly
+// queue up at the same few L2 lines.  Instead a CTA copies both masks to shared memory once per sweep,
+// its warps decide what they can from the copy and publish decisions with atomics; a decision reaches the
+// other CTAs with their next copy.
 //
-// One cooperative kernel (every CTA resident), 256 threads, three parts:
+// One cooperative kernel (every CTA resident), one CTA of 1024 threads per SM, three parts:
 //  1. "earlier" is decided from the integer densities themselves (no rank array): the densities of an
 //     image are staged in shared memory, each warp masks the adjacency words of its rows down to the
-//     earlier neighbours (written back, and the first row's words stay in registers);
-//  2. resolution loop (bounded);
+//     earlier neighbours (the first row's words stay in registers, further rows are written back);
+//  2. sweeps (bounded) until no row of the CTA is pending;
 //  3. after a grid-wide barrier: cluster ids (number of centres with a lower index), centre list,
 //     centre keys and inverse norms.
 constexpr int kAdjRegs = 8;      // adjacency words per lane kept in registers: rows of up to 8192 survivors
+constexpr int kCenThreads = 1024;
+constexpr int kCenWarps = kCenThreads / 32;
 
 template <typename T>
-__global__ void __launch_bounds__(256) k_centers(const __grid_constant__ Batch bt, int keys_cap, int spin_limit) {
+__global__ void __launch_bounds__(kCenThreads, 1) k_centers(const __grid_constant__ Batch bt, int keys_cap, int mask_cap,
+                                                            int spin_limit) {
   using D = typename DistOf<T>::type;
   constexpr int V = Vec<T>::N;
   cooperative_groups::grid_group grid = cooperative_groups::this_grid();
   TL_SCOPE(bt.img[0], 5);
   extern __shared__ unsigned long long skeys[];          // [keys_cap] densities of this CTA's image
-  const int lane = threadIdx.x & 31;
+  uint32_t *cm_s = reinterpret_cast<uint32_t *>(skeys + keys_cap);   // [mask_cap] copy of the centre mask
+  uint32_t *rm_s = cm_s + mask_cap;                      // [mask_cap] copy of the removed mask
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   // The CTAs are shared out evenly among the images (the last image also takes the remainder); a CTA
   // works on one image throughout, so the images of a batch are resolved side by side.
-  const int per = gridDim.x / bt.B;
+  const int per = max(1, (int)gridDim.x / bt.B);
   const int b = min((int)blockIdx.x / per, bt.B - 1);
   const int ncta = b == bt.B - 1 ? (int)gridDim.x - per * (bt.B - 1) : per;
-  const int nwarps = ncta * 8;
-  const int gw = ((int)blockIdx.x - b * per) * 8 + (threadIdx.x >> 5);
+  const int nwarps = ncta * kCenWarps;
+  const int gw = ((int)blockIdx.x - b * per) * kCenWarps + wid;
   const ImgDesc &im = bt.img[b];
+  pdl_wait();
+  pdl_trigger();
   const int q = *im.q_ptr, nw = (q + 31) >> 5;
 
   // part 1: keep only the neighbours that come earlier in density order
@@ -322,7 +332,7 @@ __global__ void __launch_bounds__(256) k_centers(const __grid_constant__ Batch b
   {
     const bool in_smem = q <= keys_cap;
     if (in_smem)
-      for (int r = threadIdx.x; r < q; r += 256) skeys[r] = im.rho_fix[r];
+      for (int r = threadIdx.x; r < q; r += kCenThreads) skeys[r] = im.rho_fix[r];
     __syncthreads();
     const unsigned long long *keys = in_smem ? skeys : im.rho_fix;
     for (int r = gw; r < q; r += nwarps) {
@@ -343,7 +353,7 @@ __global__ void __launch_bounds__(256) k_centers(const __grid_constant__ Batch b
           const unsigned long long o = keys[j];
           if (j != r && (o > mine || (o == mine && j < r))) out |= 1u << bpos;
         }
-        if (wd < nw) row[wd] = out;
+        if (wd < nw && !keep_regs) row[wd] = out;
         if (keep_regs) cached[u] = out;
       }
       for (int wd = lane + 32 * kAdjRegs; wd < nw; wd += 32) {     // rows longer than the register part
@@ -365,41 +375,45 @@ __global__ void __launch_bounds__(256) k_centers(const __grid_constant__ Batch b
       }
     }
   }
-  __syncwarp();
   TL_POINT(bt.img[0], 10);
 
   // part 2: resolve
-  int sweeps = 0, pending = 1;
+  const bool masks_in_smem = nw <= mask_cap;
+  int sweeps = 0;
   bool cached_done = false;
-  while (pending && sweeps < spin_limit) {
-    pending = 0;
+  for (;;) {
+    if (masks_in_smem) {
+      __syncthreads();                                  // the previous sweep has read the copy
+      for (int wd = threadIdx.x; wd < nw; wd += kCenThreads) {
+        cm_s[wd] = ld_relaxed_u32(&im.cmask[wd]);
+        rm_s[wd] = ld_relaxed_u32(&im.rmask[wd]);
+      }
+      __syncthreads();
+    }
+    const uint32_t *cmL = masks_in_smem ? cm_s : im.cmask, *rmL = masks_in_smem ? rm_s : im.rmask;
+    auto ldm = [&](const uint32_t *p) { return masks_in_smem ? *p : ld_relaxed_u32(p); };
+    int pending = 0;
     ++sweeps;
     for (int r = gw; r < q; r += nwarps) {
       const uint32_t mybit = 1u << (r & 31);
       bool hit_center = false, alive = false;
       if (r == cached_item) {                     // the masked adjacency of this row is in registers
         if (cached_done) continue;
-        uint32_t cm[kAdjRegs], rm[kAdjRegs];
 #pragma unroll
         for (int u = 0; u < kAdjRegs; ++u) {
-          const bool need = cached[u] != 0u;
-          cm[u] = need ? ld_relaxed_u32(&im.cmask[lane + 32 * u]) : 0u;
-          rm[u] = need ? ld_relaxed_u32(&im.rmask[lane + 32 * u]) : 0u;
-        }
-#pragma unroll
-        for (int u = 0; u < kAdjRegs; ++u) {
-          hit_center |= (cached[u] & cm[u]) != 0u;
-          alive |= (cached[u] & ~rm[u]) != 0u;
+          if (cached[u] != 0u) {
+            hit_center |= (cached[u] & ldm(&cmL[lane + 32 * u])) != 0u;
+            alive |= (cached[u] & ~ldm(&rmL[lane + 32 * u])) != 0u;
+          }
         }
       } else {
-        const uint32_t decided = (ld_relaxed_u32(&im.cmask[r >> 5]) | ld_relaxed_u32(&im.rmask[r >> 5])) & mybit;
-        if (decided) continue;
+        if ((ldm(&cmL[r >> 5]) | ldm(&rmL[r >> 5])) & mybit) continue;   // decided
         const uint32_t *row = im.adj + (size_t)r * im.Wp;
         for (int wd = lane; wd < nw; wd += 32) {
           const uint32_t e = row[wd];
           if (e) {
-            hit_center |= (e & ld_relaxed_u32(&im.cmask[wd])) != 0u;
-            alive |= (e & ~ld_relaxed_u32(&im.rmask[wd])) != 0u;
+            hit_center |= (e & ldm(&cmL[wd])) != 0u;
+            alive |= (e & ~ldm(&rmL[wd])) != 0u;
           }
         }
       }
@@ -415,12 +429,13 @@ __global__ void __launch_bounds__(256) k_centers(const __grid_constant__ Batch b
         pending = 1;
       }
     }
-    if (pending) __nanosleep(100);                 // the masks are polled by thousands of warps: do not hammer them
+    if (!__syncthreads_or(pending)) break;              // no row of this CTA is pending
+    if (sweeps >= spin_limit) {
+      if (threadIdx.x == 0) atomicMin(&im.cnt[PACT_CNT_STATUS], (int)PACT_ERR_TIMEOUT);
+      break;
+    }
   }
-  if (lane == 0 && gw < q) {
-    if (pending) atomicMin(&im.cnt[PACT_CNT_STATUS], (int)PACT_ERR_TIMEOUT);
-    atomicMax(&im.cnt[PACT_CNT_SWEEPS], sweeps);
-  }
+  if (threadIdx.x == 0 && gw < q) atomicMax(&im.cnt[PACT_CNT_SWEEPS], sweeps);
 
   // part 3: every decision is final once all CTAs are here
   TL_POINT(bt.img[0], 11);
@@ -428,10 +443,9 @@ __global__ void __launch_bounds__(256) k_centers(const __grid_constant__ Batch b
   grid.sync();
   TL_POINT(bt.img[0], 12);
   // Cluster id of a centre = number of centres with a lower index.  The centre mask of an image is read
-  // once per CTA into shared memory with its running bit counts (every warp reading the same few words
-  // from global memory makes them a hot spot); images too large for the staging buffer take the words
-  // from global memory.
-  __shared__ int wsum3[8];
+  // once per CTA into shared memory with its running bit counts; images too large for the staging buffer
+  // take the words from global memory.
+  __shared__ int wsum3[kCenWarps];
   __shared__ int s_carry3;
   {
     const bool staged = q <= keys_cap;              // nw words and nw counts fit where the densities were
@@ -441,7 +455,7 @@ __global__ void __launch_bounds__(256) k_centers(const __grid_constant__ Batch b
     if (staged) {
       if (threadIdx.x == 0) s_carry3 = 0;
       __syncthreads();
-      for (int base = 0; base < nw; base += 256) {
+      for (int base = 0; base < nw; base += kCenThreads) {
         const int wd = base + threadIdx.x;
         const uint32_t m = wd < nw ? __ldcg(&im.cmask[wd]) : 0u;
         const int pc = __popc(m);
@@ -451,13 +465,13 @@ __global__ void __launch_bounds__(256) k_centers(const __grid_constant__ Batch b
           const int y = __shfl_up_sync(0xffffffffu, x, o);
           if (lane >= o) x += y;
         }
-        if (lane == 31) wsum3[threadIdx.x >> 5] = x;
+        if (lane == 31) wsum3[wid] = x;
         __syncthreads();
         int off = s_carry3;
-        for (int k = 0; k < (int)(threadIdx.x >> 5); ++k) off += wsum3[k];
+        for (int k = 0; k < wid; ++k) off += wsum3[k];
         if (wd < nw) { cm[wd] = m; pref[wd] = off + x - pc; }
         __syncthreads();
-        if (threadIdx.x == 255) s_carry3 = off + x;
+        if (threadIdx.x == kCenThreads - 1) s_carry3 = off + x;
         __syncthreads();
       }
     }
@@ -655,21 +669,22 @@ void launch_gram(const Batch &bt, int maxN, bool bf16, const ClusterCfg &cfg, cu
 }
 
 cudaError_t launch_centers(const Batch &bt, int maxQ, bool bf16, const ClusterCfg &cfg, int spin_limit, cudaStream_t st) {
-  // the densities of one image are staged in shared memory when they fit in a quarter of it; maxQ is
-  // an estimate of the largest survivor count, an image with more reads them from global memory
-  size_t smem = (size_t)maxQ * sizeof(unsigned long long);
-  const size_t budget = (size_t)cfg.centers_smem_max / 4;
-  if (smem > budget) smem = 0;
-  int keys_cap = (int)(smem / sizeof(unsigned long long));
+  // the densities of one image are staged in shared memory when they fit in half of it; maxQ is an estimate of
+  // the largest survivor count, an image with more reads them from global memory.  The two mask copies
+  // take a word per 32 survivors each.
+  const size_t budget = (size_t)cfg.centers_smem_max / 2;
+  int keys_cap = (size_t)maxQ * sizeof(unsigned long long) <= budget ? maxQ : 0;
+  int mask_cap = (maxQ + 31) / 32 + 1;
+  if ((size_t)mask_cap * 8 > budget) mask_cap = 0;
+  const size_t smem = (size_t)keys_cap * sizeof(unsigned long long) + (size_t)mask_cap * 8;
   const void *fn = bf16 ? (const void *)k_centers<__nv_bfloat16> : (const void *)k_centers<float>;
   int per_sm = 0;
-  cudaError_t e = bf16 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_centers<__nv_bfloat16>, 256, smem)
-                       : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_centers<float>, 256, smem);
+  cudaError_t e = bf16 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_centers<__nv_bfloat16>, kCenThreads, smem)
+                       : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_centers<float>, kCenThreads, smem);
   if (e != cudaSuccess) return e;
   if (per_sm < 1) return cudaErrorLaunchOutOfResources;
-  if (per_sm > 4) per_sm = 4;
-  void *args[] = {(void *)&bt, (void *)&keys_cap, (void *)&spin_limit};
-  return cudaLaunchCooperativeKernel(fn, dim3(cfg.sm_count * per_sm), dim3(256), args, smem, st);
+  void *args[] = {(void *)&bt, (void *)&keys_cap, (void *)&mask_cap, (void *)&spin_limit};
+  return cudaLaunchCooperativeKernel(fn, dim3(cfg.sm_count), dim3(kCenThreads), args, smem, st);
 }
 
 void launch_assign(const Batch &bt, int maxN, bool bf16, RowMode mode, const ClusterCfg &cfg, cudaStream_t st) {
