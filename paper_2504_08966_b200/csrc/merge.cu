@@ -40,9 +40,7 @@ template <> __device__ __forceinline__ void store_vec8<__nv_bfloat16>(__nv_bfloa
 template <typename T> struct Raw8;
 template <> struct Raw8<__nv_bfloat16> {
   uint4 a;
-  __device__ __forceinline__ void load(const __nv_bfloat16 *p, unsigned long long pol) {
-    a = ldg_hint(reinterpret_cast<const uint4 *>(p), pol);
-  }
+  __device__ __forceinline__ void from_ring(const uint4 *p) { a = p[0]; }
   __device__ __forceinline__ void add_to(float (&acc)[8]) const {
     float x[8];
     widen_vec<__nv_bfloat16>(a, x);
@@ -52,10 +50,7 @@ template <> struct Raw8<__nv_bfloat16> {
 };
 template <> struct Raw8<float> {
   uint4 a, b;
-  __device__ __forceinline__ void load(const float *p, unsigned long long pol) {
-    a = ldg_hint(reinterpret_cast<const uint4 *>(p), pol);
-    b = ldg_hint(reinterpret_cast<const uint4 *>(p) + 1, pol);
-  }
+  __device__ __forceinline__ void from_ring(const uint4 *p) { a = p[0]; b = p[1]; }
   __device__ __forceinline__ void add_to(float (&acc)[8]) const {
     float x[4], y[4];
     widen_vec<float>(a, x);
@@ -268,19 +263,22 @@ __global__ void __launch_bounds__(kListBlock) k_lists(const __grid_constant__ Ba
 }
 
 // ---- Eq. 10 ------------------------------------------------------------------------------------------
-// Grid (X, B), kMrgThreads threads, one CTA per SM.  Work items are the member records in cluster order
+// Grid (X, B), kMrgThreads threads, two CTAs per SM.  Work items are the member records in cluster order
 // followed by the text rows; CTA x takes items [x per, (x + 1) per).  A thread owns VPL groups of 8 columns
-// and adds the rows of the running cluster in float; the loads of the next R rows are issued before the
-// current R rows are added.  A cluster that lies inside the range is divided and stored when the next one
-// begins.  A range boundary cuts at most two clusters per CTA: the one that began before the range (its
+// and adds the rows of the running cluster in float.  The rows arrive through a ring of DEPTH rows in shared
+// memory filled with asynchronous 16-byte copies (every thread copies and later reads its own columns, so
+// the ring needs no barrier): DEPTH rows are in flight per SM whatever the registers hold.  A cluster that
+// lies inside the range is divided and stored when the next one begins.  A range boundary cuts at most two clusters per CTA: the one that began before the range (its
 // sum is set aside when it ends) and the one that goes on after it.  Their sums go to scratch (slot 0 and
 // slot 1 of the CTA) with a ticket each; the CTA that draws a cluster's last ticket adds the sums in range
 // order and stores the row, so the result does not depend on which CTA that is.
 constexpr int kMrgThreads = 512;
-constexpr int kMrgTile = 64;                        // records staged in shared memory at a time
+constexpr int kMrgTile = 256;                       // records staged in shared memory at a time
+constexpr int kMrgCtasPerSm = 2;
+constexpr int kMrgRingBytes = 160 * 1024 / kMrgCtasPerSm;   // rows in flight per CTA
 
-template <typename T, typename O, int VPL, int R>
-__global__ void __launch_bounds__(kMrgThreads, 1) k_merge(const __grid_constant__ Batch bt) {
+template <typename T, typename O, int VPL, int DEPTH>
+__global__ void __launch_bounds__(kMrgThreads, kMrgCtasPerSm) k_merge(const __grid_constant__ Batch bt) {
   const ImgDesc &im = bt.img[blockIdx.y];
   TL_SCOPE(im, 9);
   const int t = threadIdx.x;
@@ -300,18 +298,15 @@ __global__ void __launch_bounds__(kMrgThreads, 1) k_merge(const __grid_constant_
   const int per = (total + X - 1) / X;
   const int lo = min(total, x * per), hi = min(total, lo + per);
   if (x == 0 && t == 0) im.cnt[PACT_CNT_N_OUT] = n_text + C;
-  const unsigned long long pol_last_use = policy_evict_first();   // the rows are not read again
 
-  float acc[VPL][8], head[VPL][8];
+  float acc[VPL][8];
   int cur_c = -1, cur_off = 0, cur_size = 0, cur_dst = 0;
   float cur_inv = 1.f;
-  int head_c = -1, head_off = 0, head_size = 0, head_dst = 0;   // the cluster that began before this range
-  float head_inv = 1.f;
-  bool head_open = false;                           // the running cluster is that one
+  bool head_open = false;                           // the running cluster began before this range
 #pragma unroll
   for (int v = 0; v < VPL; ++v)
 #pragma unroll
-    for (int e = 0; e < 8; ++e) { acc[v][e] = 0.f; head[v][e] = 0.f; }
+    for (int e = 0; e < 8; ++e) acc[v][e] = 0.f;
 
   auto store_row = [&](const float (&a)[VPL][8], float inv, int dst) {
 #pragma unroll
@@ -322,54 +317,6 @@ __global__ void __launch_bounds__(kMrgThreads, 1) k_merge(const __grid_constant_
 #pragma unroll
         for (int e = 0; e < 8; ++e) y[e] = a[v][e] * inv;
         store_vec8<O>(Ho + (size_t)dst * im.ldHo + g * 8, y);
-      }
-    }
-  };
-  auto issue = [&](Raw8<T> (&xr)[R][VPL], int j0, int tn) {
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-      if (j0 + r < tn) {
-        const T *row = H + (size_t)s_rec[j0 + r].x * im.ldH;
-#pragma unroll
-        for (int v = 0; v < VPL; ++v) {
-          const int g = t + v * kMrgThreads;
-          if (g < ng) xr[r][v].load(row + g * 8, pol_last_use);
-        }
-      }
-    }
-  };
-  auto consume = [&](const Raw8<T> (&xr)[R][VPL], int j0, int tn) {
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-      if (j0 + r < tn) {
-        const int4 rec = s_rec[j0 + r];
-        if (rec.y != cur_c) {                        // the next cluster begins (the same for all threads)
-          if (cur_c >= 0) {
-            if (head_open) {
-#pragma unroll
-              for (int v = 0; v < VPL; ++v)
-#pragma unroll
-                for (int e = 0; e < 8; ++e) head[v][e] = acc[v][e];
-              head_c = cur_c; head_off = cur_off; head_size = cur_size; head_dst = cur_dst; head_inv = cur_inv;
-              head_open = false;
-            } else {
-              store_row(acc, cur_inv, cur_dst);
-            }
-          } else {
-            head_open = rec.z < lo;
-          }
-#pragma unroll
-          for (int v = 0; v < VPL; ++v)
-#pragma unroll
-            for (int e = 0; e < 8; ++e) acc[v][e] = 0.f;
-          cur_c = rec.y; cur_off = rec.z; cur_size = rec.w;
-          cur_dst = s_dst[j0 + r]; cur_inv = s_inv[j0 + r];
-        }
-#pragma unroll
-        for (int v = 0; v < VPL; ++v) {
-          const int g = t + v * kMrgThreads;
-          if (g < ng) xr[r][v].add_to(acc[v]);
-        }
       }
     }
   };
@@ -413,6 +360,59 @@ __global__ void __launch_bounds__(kMrgThreads, 1) k_merge(const __grid_constant_
     store_row(a, inv, dst);
   };
 
+  constexpr int Q16 = (int)sizeof(T) * 8 / 16;        // 16-byte pieces of a group of 8 columns
+  constexpr int kSlot = VPL * kMrgThreads * Q16;      // 16-byte pieces per ring slot
+  extern __shared__ uint4 ring[];                     // [DEPTH][kSlot]
+  auto issue = [&](int j, int tn) {                   // row j of the tile -> slot j % DEPTH; one group per call
+    if (j < tn) {
+      const T *row = H + (size_t)s_rec[j].x * im.ldH;
+      uint4 *slot = ring + (size_t)(j % DEPTH) * kSlot;
+#pragma unroll
+      for (int v = 0; v < VPL; ++v) {
+        const int g = t + v * kMrgThreads;
+        if (g < ng) {
+#pragma unroll
+          for (int pc = 0; pc < Q16; ++pc) {
+            const unsigned dsta = (unsigned)__cvta_generic_to_shared(slot + (size_t)g * Q16 + pc);
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dsta), "l"(row + g * 8 + pc * (16 / (int)sizeof(T))) : "memory");
+          }
+        }
+      }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  auto consume = [&](int j) {
+    asm volatile("cp.async.wait_group %0;" ::"n"(DEPTH - 1) : "memory");
+    const int4 rec = s_rec[j];
+    if (rec.y != cur_c) {                            // the next cluster begins (the same for all threads)
+      if (cur_c >= 0) {
+        if (head_open) {                               // the cluster that began before this range ends here
+          cut(acc, cur_c, cur_off, cur_size, cur_inv, cur_dst, 0);
+          head_open = false;
+        } else {
+          store_row(acc, cur_inv, cur_dst);
+        }
+      } else {
+        head_open = rec.z < lo;
+      }
+#pragma unroll
+      for (int v = 0; v < VPL; ++v)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[v][e] = 0.f;
+      cur_c = rec.y; cur_off = rec.z; cur_size = rec.w;
+      cur_dst = s_dst[j]; cur_inv = s_inv[j];
+    }
+    const uint4 *slot = ring + (size_t)(j % DEPTH) * kSlot;
+#pragma unroll
+    for (int v = 0; v < VPL; ++v) {
+      const int g = t + v * kMrgThreads;
+      if (g < ng) {
+        Raw8<T> x;
+        x.from_ring(slot + (size_t)g * Q16);
+        x.add_to(acc[v]);
+      }
+    }
+  };
   for (int t0 = lo; t0 < hi; t0 += kMrgTile) {
     const int tn = min(kMrgTile, hi - t0);
     __syncthreads();                                 // the previous tile's records are no longer needed
@@ -445,14 +445,11 @@ __global__ void __launch_bounds__(kMrgThreads, 1) k_merge(const __grid_constant_
       s_inv[t] = inv;
     }
     __syncthreads();
-    Raw8<T> xa[R][VPL], xb[R][VPL];
-    issue(xa, 0, tn);
+    for (int j = 0; j < DEPTH; ++j) issue(j, tn);
 #pragma unroll 1
-    for (int j0 = 0; j0 < tn; j0 += 2 * R) {
-      if (j0 + R < tn) issue(xb, j0 + R, tn);
-      consume(xa, j0, tn);
-      if (j0 + 2 * R < tn) issue(xa, j0 + 2 * R, tn);
-      if (j0 + R < tn) consume(xb, j0 + R, tn);
+    for (int j = 0; j < tn; ++j) {
+      consume(j);
+      issue(j + DEPTH, tn);
     }
   }
   if (cur_c < 0) return;                             // an empty range
@@ -461,7 +458,6 @@ __global__ void __launch_bounds__(kMrgThreads, 1) k_merge(const __grid_constant_
     cut(acc, cur_c, cur_off, cur_size, cur_inv, cur_dst, goes_on ? 1 : 0);
     return;
   }
-  if (head_c >= 0) cut(head, head_c, head_off, head_size, head_inv, head_dst, 0);
   if (goes_on) cut(acc, cur_c, cur_off, cur_size, cur_inv, cur_dst, 1);
   else store_row(acc, cur_inv, cur_dst);
 }
@@ -498,17 +494,29 @@ int lists_kernels(int maxN, int B) {
 }
 
 int merge_ctas(int sm_count, int B) {
-  const int X = sm_count / B;
+  const int X = kMrgCtasPerSm * sm_count / B;
   return X < 1 ? 1 : X;
+}
+
+template <typename T, typename O, int VPL>
+static cudaError_t launch_merge_v(const Batch &bt, dim3 grid, cudaStream_t st) {
+  constexpr int kSlotBytes = VPL * kMrgThreads * 8 * (int)sizeof(T);
+  constexpr int DEPTH = kMrgRingBytes / kSlotBytes;
+  return launch_k(k_merge<T, O, VPL, DEPTH>, grid, dim3(kMrgThreads), (size_t)DEPTH * kSlotBytes, st, false, bt);
 }
 
 template <typename T, typename O>
 static cudaError_t launch_merge_t(const Batch &bt, const ClusterCfg &cfg, cudaStream_t st) {
   dim3 grid(merge_ctas(cfg.sm_count, bt.B), bt.B);
-  constexpr int R1 = sizeof(T) == 2 ? 8 : 4;         // rows per batch; two batches are in flight
-  if (bt.d <= kMrgThreads * 8) k_merge<T, O, 1, R1><<<grid, kMrgThreads, 0, st>>>(bt);
-  else k_merge<T, O, kMergeMaxD / 8 / kMrgThreads, R1 / 2><<<grid, kMrgThreads, 0, st>>>(bt);
-  return cudaGetLastError();
+  if (bt.d <= kMrgThreads * 8) return launch_merge_v<T, O, 1>(bt, grid, st);
+  return launch_merge_v<T, O, kMergeMaxD / 8 / kMrgThreads>(bt, grid, st);
+}
+
+template <typename T, typename O, int VPL>
+static cudaError_t merge_attr() {
+  constexpr int kSlotBytes = VPL * kMrgThreads * 8 * (int)sizeof(T);
+  constexpr int DEPTH = kMrgRingBytes / kSlotBytes;
+  return cudaFuncSetAttribute(k_merge<T, O, VPL, DEPTH>, cudaFuncAttributeMaxDynamicSharedMemorySize, DEPTH * kSlotBytes);
 }
 
 cudaError_t merge_configure() {
@@ -527,7 +535,16 @@ cudaError_t merge_configure() {
   if (e != cudaSuccess) return e;
   m = per_sm < m ? per_sm : m;
   g_lists_resident = m * sms;
-  return cudaSuccess;
+  constexpr int V2 = kMergeMaxD / 8 / kMrgThreads;
+  e = merge_attr<__nv_bfloat16, __nv_bfloat16, 1>();
+  if (e == cudaSuccess) e = merge_attr<__nv_bfloat16, __nv_bfloat16, V2>();
+  if (e == cudaSuccess) e = merge_attr<__nv_bfloat16, float, 1>();
+  if (e == cudaSuccess) e = merge_attr<__nv_bfloat16, float, V2>();
+  if (e == cudaSuccess) e = merge_attr<float, __nv_bfloat16, 1>();
+  if (e == cudaSuccess) e = merge_attr<float, __nv_bfloat16, V2>();
+  if (e == cudaSuccess) e = merge_attr<float, float, 1>();
+  if (e == cudaSuccess) e = merge_attr<float, float, V2>();
+  return e;
 }
 
 cudaError_t launch_merge(const Batch &bt, bool in_bf16, bool out_bf16, const ClusterCfg &cfg, cudaStream_t st) {
