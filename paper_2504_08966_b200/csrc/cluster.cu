@@ -677,14 +677,13 @@ cudaError_t launch_centers(const Batch &bt, int maxQ, bool bf16, const ClusterCf
   int mask_cap = (maxQ + 31) / 32 + 1;
   if ((size_t)mask_cap * 8 > budget) mask_cap = 0;
   const size_t smem = (size_t)keys_cap * sizeof(unsigned long long) + (size_t)mask_cap * 8;
-  const void *fn = bf16 ? (const void *)k_centers<__nv_bfloat16> : (const void *)k_centers<float>;
   int per_sm = 0;
   cudaError_t e = bf16 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_centers<__nv_bfloat16>, kCenThreads, smem)
                        : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_centers<float>, kCenThreads, smem);
   if (e != cudaSuccess) return e;
   if (per_sm < 1) return cudaErrorLaunchOutOfResources;
-  void *args[] = {(void *)&bt, (void *)&keys_cap, (void *)&mask_cap, (void *)&spin_limit};
-  return cudaLaunchCooperativeKernel(fn, dim3(cfg.sm_count), dim3(kCenThreads), args, smem, st);
+  return bf16 ? launch_coop(k_centers<__nv_bfloat16>, dim3(cfg.sm_count), dim3(kCenThreads), smem, st, true, bt, keys_cap, mask_cap, spin_limit)
+              : launch_coop(k_centers<float>, dim3(cfg.sm_count), dim3(kCenThreads), smem, st, true, bt, keys_cap, mask_cap, spin_limit);
 }
 
 void launch_assign(const Batch &bt, int maxN, bool bf16, RowMode mode, const ClusterCfg &cfg, cudaStream_t st) {

@@ -239,6 +239,127 @@ __device__ __forceinline__ void gram_chunk(const uint32_t (&v)[32], const float 
   }
 }
 
+// The epilogue of one accumulator tile for one warp: the warp's 32 rows (tensor-memory lanes) of the 128-row
+// block tmi against HALF columns from cbase on.  Waits for the accumulator, reads it 32 columns at a time and
+// applies the mode's arithmetic; arrive() is called once the accumulator has been read.  skip: the warp only
+// waits and releases (a block below the diagonal of the all-pairs pass).  Returns false when the wait ran out.
+template <int MODE, int HALF, typename Arrive>
+__device__ __forceinline__ bool epi_tile(const ImgDesc &im, int kept_rows, int tmi, int cbase, bool skip, int nrows,
+                                         int ncols, uint32_t taddr, uint64_t *acc_full, uint32_t parity, float *rn_col,
+                                         uint32_t *tr, int lane, int qd, int &band, float &mx, Arrive arrive) {
+  // inverse norms of this warp's columns and of this lane's row (in flight while the MMAs run)
+  const float *rn_src = MODE == MODE_GRAM ? im.rnk : (MODE == MODE_SPREAD ? im.rn : im.rnc);
+  float4 r4;
+  {
+    const int gj = cbase + lane * 4;
+    r4.x = gj + 0 < ncols ? rn_src[gj + 0] : 0.f;
+    r4.y = gj + 1 < ncols ? rn_src[gj + 1] : 0.f;
+    r4.z = gj + 2 < ncols ? rn_src[gj + 2] : 0.f;
+    r4.w = gj + 3 < ncols ? rn_src[gj + 3] : 0.f;
+  }
+  const int row = tmi * BM + qd * 32 + lane;
+  const bool row_ok = row < nrows;
+  const bool kept_space = MODE == MODE_GRAM || (MODE == MODE_ASSIGN && kept_rows);
+  float rni = row_ok ? (kept_space ? im.rnk[row] : im.rn[row]) : 0.f;
+  if (MODE == MODE_GRAM) {
+    // the all-pairs pass multiplies the two inverse norms first; a vanishing key (inverse norm at
+    // its clamp, 1e20) takes 0 here so that the product stays finite: dot product 0, distance 1
+    constexpr float kHuge = 1e19f;
+    if (rni > kHuge) rni = 0.f;
+    if (r4.x > kHuge) r4.x = 0.f;
+    if (r4.y > kHuge) r4.y = 0.f;
+    if (r4.z > kHuge) r4.z = 0.f;
+    if (r4.w > kHuge) r4.w = 0.f;
+  }
+  __syncwarp();
+  if (lane * 4 < HALF) reinterpret_cast<float4 *>(rn_col)[lane] = r4;
+  __syncwarp();
+  if (!mbar_wait_warp(acc_full, parity)) return false;
+  tc_fence_after();
+  unsigned long long rowsum = 0ull;
+  float bd = 3.0f;                              // best distance so far (assignment); distances are <= 2
+  int bi = 0;
+  const float d_c = im.d_c, neg_k = -im.inv_dn_log2e;
+  const int r0 = tmi * BM + qd * 32;
+  const bool above = MODE == MODE_GRAM && cbase / BM > tmi;   // block above the diagonal: rows and columns
+#pragma unroll 1
+  for (int ch = 0; ch < HALF / 32; ++ch) {
+    const int c0 = cbase + ch * 32;
+    if (skip || c0 >= ncols) break;              // uniform
+    uint32_t v[32];
+    tmem_ld32(taddr + ch * 32, v);
+    tmem_ld_wait();
+    if (MODE == MODE_GRAM) {
+      uint32_t bits, colbits = 0u;
+      unsigned long long colsum = 0ull;
+      if (above) {
+        // every row of this block is a survivor (only the last block row is ragged, and it has no
+        // block to its right); each pair (row, column) is also the pair (column, row)
+        int bnd = 0;
+        if (c0 + 32 > ncols)
+          gram_chunk<true, true>(v, rn_col + ch * 32, rni, row, c0, ncols, d_c, neg_k, lane, tr, rowsum, bits, bnd, colsum, colbits);
+        else
+          gram_chunk<false, true>(v, rn_col + ch * 32, rni, row, c0, ncols, d_c, neg_k, lane, tr, rowsum, bits, bnd, colsum, colbits);
+        band += bnd;                            // row < column throughout
+        const int gj = c0 + lane;
+        if (gj < ncols) {
+          atomicAdd(&im.rho_fix[gj], colsum);
+          im.adj[(size_t)gj * im.Wp + (r0 >> 5)] = colbits;
+        }
+      } else {
+        const bool edge = (c0 + 32 > ncols) || (c0 < r0 + 32 && c0 + 32 > r0);
+        if (edge) gram_chunk<true, false>(v, rn_col + ch * 32, rni, row, c0, ncols, d_c, neg_k, lane, tr, rowsum, bits, band, colsum, colbits);
+        else {
+          int bnd = 0;
+          gram_chunk<false, false>(v, rn_col + ch * 32, rni, row, c0, ncols, d_c, neg_k, lane, tr, rowsum, bits, bnd, colsum, colbits);
+          if (row < c0) band += bnd;            // each unordered pair once; the chunk lies wholly on one side
+        }
+      }
+      if (row_ok) im.adj[(size_t)row * im.Wp + (c0 >> 5)] = bits;
+    } else if (MODE == MODE_SPREAD) {
+      // rows and columns past the end hold zero dot products, i.e. distance 1: leave them out
+      const int lim = row_ok ? min(32, ncols - c0) : 0;
+      const int self = row - c0;                 // the pair (i, i) is not a pair
+#pragma unroll
+      for (int k4 = 0; k4 < 32; k4 += 4) {
+        const float4 rn4 = *reinterpret_cast<const float4 *>(rn_col + ch * 32 + k4);
+        const float rnj[4] = {rn4.x, rn4.y, rn4.z, rn4.w};
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+          const int k = k4 + kk;
+          const float dd = DistF::dist(__uint_as_float(v[k]), rni, rnj[kk]);
+          if (k < lim && k != self) mx = fmaxf(mx, dd);
+        }
+      }
+    } else {
+      const int lim = min(32, ncols - c0);
+#pragma unroll
+      for (int k4 = 0; k4 < 32; k4 += 4) {
+        const float4 rn4 = *reinterpret_cast<const float4 *>(rn_col + ch * 32 + k4);
+        const float rnj[4] = {rn4.x, rn4.y, rn4.z, rn4.w};
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+          const int k = k4 + kk;
+          const float dd = DistF::dist(__uint_as_float(v[k]), rni, rnj[kk]);
+          if (k < lim && dd < bd) { bd = dd; bi = c0 + k; }
+        }
+      }
+    }
+  }
+  // the accumulator may be overwritten once all epilogue warps have read it
+  tc_fence_before();
+  __syncwarp();
+  if (lane == 0) arrive();
+  if (row_ok && !skip) {
+    if (MODE == MODE_GRAM) atomicAdd(&im.rho_fix[row], rowsum);
+    else if (MODE == MODE_ASSIGN && bd <= 2.0f) {
+      const unsigned long long pk = ((unsigned long long)__float_as_uint(bd) << 32) | (unsigned)bi;
+      atomicMin(&im.best[kept_rows ? im.kept_idx[row] : row], pk);
+    }
+  }
+  return true;
+}
+
 }  // namespace
 
 // grid (X, B), 320 threads, dynamic smem = TileCfg<BN>::SMEM.
@@ -257,15 +378,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
   uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-  int nrows, ncols;
-  if (MODE == MODE_GRAM) { nrows = *im.q_ptr; ncols = nrows; }
-  else if (MODE == MODE_SPREAD) { nrows = im.N; ncols = im.N; }
-  else { nrows = kept_rows ? *im.q_ptr : im.N; ncols = *im.C_ptr; }
-  const int ntm = (nrows + BM - 1) / BM, ntn = (ncols + BN - 1) / BN;
-  const int ntiles = tile_count<MODE>(ntm, ntn);
-  if ((int)blockIdx.x >= ntiles) return;            // uniform: nothing allocated yet
-  const int nslab = bt.d_k / BK;
-
+  // set-up that does not depend on the kernels before this one
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
     for (int a = 0; a < NACC; ++a) { mbar_init(&sh.acc_full[a], 1); mbar_init(&sh.acc_empty[a], EPI_WARPS); }
@@ -277,8 +390,20 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = sh.tmem_base;
+  pdl_wait();
+  pdl_trigger();
 
-  if (warp == 0) {
+  int nrows, ncols;
+  if (MODE == MODE_GRAM) { nrows = *im.q_ptr; ncols = nrows; }
+  else if (MODE == MODE_SPREAD) { nrows = im.N; ncols = im.N; }
+  else { nrows = kept_rows ? *im.q_ptr : im.N; ncols = *im.C_ptr; }
+  const int ntm = (nrows + BM - 1) / BM, ntn = (ncols + BN - 1) / BN;
+  const int ntiles = tile_count<MODE>(ntm, ntn);
+  const bool active = (int)blockIdx.x < ntiles;       // CTAs without a tile only give their tensor memory back
+  const int nslab = bt.d_k / BK;
+
+  if (!active) {
+  } else if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
       const CUtensorMap *ma = &tm.a[blockIdx.y], *mb = &tm.b[blockIdx.y];
@@ -355,118 +480,11 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
       if (!tile_wanted<MODE, BN>(tmi, tni)) continue;
       const uint32_t a = tcount % NACC;
       const int cbase = tni * BN + half * HALF;     // first column of this warp
-      // inverse norms of this warp's columns and of this lane's row (in flight while the MMAs run)
-      const float *rn_src = MODE == MODE_GRAM ? im.rnk : (MODE == MODE_SPREAD ? im.rn : im.rnc);
-      float4 r4;
-      {
-        const int gj = cbase + lane * 4;
-        r4.x = gj + 0 < ncols ? rn_src[gj + 0] : 0.f;
-        r4.y = gj + 1 < ncols ? rn_src[gj + 1] : 0.f;
-        r4.z = gj + 2 < ncols ? rn_src[gj + 2] : 0.f;
-        r4.w = gj + 3 < ncols ? rn_src[gj + 3] : 0.f;
-      }
-      const int row = tmi * BM + qd * 32 + lane;
-      const bool row_ok = row < nrows;
-      const bool kept_space = MODE == MODE_GRAM || (MODE == MODE_ASSIGN && kept_rows);
-      float rni = row_ok ? (kept_space ? im.rnk[row] : im.rn[row]) : 0.f;
-      if (MODE == MODE_GRAM) {
-        // the all-pairs pass multiplies the two inverse norms first; a vanishing key (inverse norm at
-        // its clamp, 1e20) takes 0 here so that the product stays finite: dot product 0, distance 1
-        constexpr float kHuge = 1e19f;
-        if (rni > kHuge) rni = 0.f;
-        if (r4.x > kHuge) r4.x = 0.f;
-        if (r4.y > kHuge) r4.y = 0.f;
-        if (r4.z > kHuge) r4.z = 0.f;
-        if (r4.w > kHuge) r4.w = 0.f;
-      }
-      __syncwarp();
-      if (lane * 4 < HALF) reinterpret_cast<float4 *>(rn_col)[lane] = r4;
-      __syncwarp();
-      if (!mbar_wait_warp(&sh.acc_full[a], (tcount / NACC) & 1)) { ok = false; break; }
-      tc_fence_after();
       const uint32_t taddr = tmem_base + a * BN + half * HALF + ((uint32_t)(qd * 32) << 16);
-      unsigned long long rowsum = 0ull;
-      float bd = 3.0f;                              // best distance so far (assignment); distances are <= 2
-      int bi = 0;
-      const float d_c = im.d_c, neg_k = -im.inv_dn_log2e;
-      const int r0 = tmi * BM + qd * 32;
-      const bool above = MODE == MODE_GRAM && tni > tmi;   // block above the diagonal: rows and columns
-#pragma unroll 1
-      for (int ch = 0; ch < HALF / 32; ++ch) {
-        const int c0 = cbase + ch * 32;
-        if (c0 >= ncols) break;                      // uniform
-        uint32_t v[32];
-        tmem_ld32(taddr + ch * 32, v);
-        tmem_ld_wait();
-        if (MODE == MODE_GRAM) {
-          uint32_t bits, colbits = 0u;
-          unsigned long long colsum = 0ull;
-          if (above) {
-            // every row of this block is a survivor (only the last block row is ragged, and it has no
-            // block to its right); each pair (row, column) is also the pair (column, row)
-            int bnd = 0;
-            if (c0 + 32 > ncols)
-              gram_chunk<true, true>(v, rn_col + ch * 32, rni, row, c0, ncols, d_c, neg_k, lane, tr, rowsum, bits, bnd, colsum, colbits);
-            else
-              gram_chunk<false, true>(v, rn_col + ch * 32, rni, row, c0, ncols, d_c, neg_k, lane, tr, rowsum, bits, bnd, colsum, colbits);
-            band += bnd;                            // row < column throughout
-            const int gj = c0 + lane;
-            if (gj < ncols) {
-              atomicAdd(&im.rho_fix[gj], colsum);
-              im.adj[(size_t)gj * im.Wp + (r0 >> 5)] = colbits;
-            }
-          } else {
-            const bool edge = (c0 + 32 > ncols) || (c0 < r0 + 32 && c0 + 32 > r0);
-            if (edge) gram_chunk<true, false>(v, rn_col + ch * 32, rni, row, c0, ncols, d_c, neg_k, lane, tr, rowsum, bits, band, colsum, colbits);
-            else {
-              int bnd = 0;
-              gram_chunk<false, false>(v, rn_col + ch * 32, rni, row, c0, ncols, d_c, neg_k, lane, tr, rowsum, bits, bnd, colsum, colbits);
-              if (row < c0) band += bnd;            // each unordered pair once; the chunk lies wholly on one side
-            }
-          }
-          if (row_ok) im.adj[(size_t)row * im.Wp + (c0 >> 5)] = bits;
-        } else if (MODE == MODE_SPREAD) {
-          // rows and columns past the end hold zero dot products, i.e. distance 1: leave them out
-          const int lim = row_ok ? min(32, ncols - c0) : 0;
-          const int self = row - c0;                 // the pair (i, i) is not a pair
-#pragma unroll
-          for (int k4 = 0; k4 < 32; k4 += 4) {
-            const float4 rn4 = *reinterpret_cast<const float4 *>(rn_col + ch * 32 + k4);
-            const float rnj[4] = {rn4.x, rn4.y, rn4.z, rn4.w};
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
-              const int k = k4 + kk;
-              const float dd = DistF::dist(__uint_as_float(v[k]), rni, rnj[kk]);
-              if (k < lim && k != self) mx = fmaxf(mx, dd);
-            }
-          }
-        } else {
-          const int lim = min(32, ncols - c0);
-#pragma unroll
-          for (int k4 = 0; k4 < 32; k4 += 4) {
-            const float4 rn4 = *reinterpret_cast<const float4 *>(rn_col + ch * 32 + k4);
-            const float rnj[4] = {rn4.x, rn4.y, rn4.z, rn4.w};
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
-              const int k = k4 + kk;
-              const float dd = DistF::dist(__uint_as_float(v[k]), rni, rnj[kk]);
-              if (k < lim && dd < bd) { bd = dd; bi = c0 + k; }
-            }
-          }
-        }
-      }
-      // the accumulator may be overwritten once all epilogue warps have read it
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&sh.acc_empty[a]);
+      ok = epi_tile<MODE, HALF>(im, kept_rows, tmi, cbase, false, nrows, ncols, taddr, &sh.acc_full[a], (tcount / NACC) & 1,
+                                rn_col, tr, lane, qd, band, mx, [&]() { mbar_arrive(&sh.acc_empty[a]); });
+      if (!ok) break;
       ++tcount;
-      if (row_ok) {
-        if (MODE == MODE_GRAM) atomicAdd(&im.rho_fix[row], rowsum);
-        else if (MODE == MODE_ASSIGN && bd <= 2.0f) {
-          const unsigned long long pk = ((unsigned long long)__float_as_uint(bd) << 32) | (unsigned)bi;
-          atomicMin(&im.best[kept_rows ? im.kept_idx[row] : row], pk);
-        }
-      }
     }
     if (!ok) atomicExch(&sh.abort, 1);
     if (MODE == MODE_GRAM && band) atomicAdd(&im.cnt[PACT_CNT_BAND_DC], band);
@@ -481,6 +499,221 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
   __syncthreads();
   tc_fence_after();
   if (warp == 1) tmem_dealloc(tmem_base, TMEM_COLS);
+  if (threadIdx.x == 0 && sh.abort) atomicMin(&im.cnt[PACT_CNT_STATUS], (int)PACT_ERR_TIMEOUT);
+}
+
+// ---- the largest-distance pass on pairs of CTAs (cta_group::2) ----------------------------------------------
+// Two CTAs of a cluster share one 256 x 256 tile: each holds 128 of its rows (operand A) and 128 of its
+// columns (half of operand B), CTA 0 issues tcgen05.mma.cta_group::2 for both, and each CTA finds its
+// 128 x 256 part of the product in its own tensor memory.  A CTA therefore fetches half as many operand
+// bytes from the L2 per output element as it does alone, and that traffic is what bounds a pass with a light
+// epilogue.  (The all-pairs pass and the rows x centres pass measured slower this way: the first is bound by
+// its epilogue, and both lose more to the coarser tiles than they gain.)
+//   full[s]      in CTA 0: both CTAs' copies of stage s report their bytes there
+//   empty[s]     in each CTA: tcgen05.commit (multicast to both CTAs) once the MMAs have read stage s
+//   acc_full[a]  in each CTA: tcgen05.commit (multicast) once accumulator a is complete
+//   acc_empty[a] in CTA 0: the epilogue warps of both CTAs arrive there
+// Every wait is bounded as in the single-CTA kernel; the CTAs leave together through a cluster barrier, after
+// which nothing is in flight towards either's shared memory.
+constexpr int PBN = 256;                              // tile width of the pair kernel
+constexpr int PSTAGES = 5;
+constexpr int PSTAGE_BYTES = 2 * A_BYTES;             // 128 rows of A and 128 rows of B per CTA and stage
+constexpr int PNACC = TMEM_COLS / PBN;
+constexpr size_t PRING = 1024 + (size_t)PSTAGES * PSTAGE_BYTES;
+template <int MODE> constexpr size_t pair_smem() { return PRING + (MODE == MODE_GRAM ? (size_t)EPI_WARPS * 32 * 36 * 4 : 0); }
+
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void cluster_barrier() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_alloc2(uint32_t *slot, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc2(uint32_t addr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+// tiled copy whose bytes are reported to a barrier that may live in the other CTA of the pair (no multicast:
+// the data go to this CTA's shared memory only)
+__device__ __forceinline__ void tma_load_2d_pair(void *dst, const CUtensorMap *map, uint32_t bar_cluster_addr, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(bar_cluster_addr), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accum) : "memory");
+}
+// arrives on the barrier at this shared-memory offset in both CTAs of the pair once the MMAs issued so far are done
+__device__ __forceinline__ void umma_commit_pair(uint64_t *bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(smem_u32(bar)), "h"((unsigned short)3) : "memory");
+}
+
+struct SharedPair {
+  uint64_t full[PSTAGES], empty[PSTAGES], acc_full[PNACC], acc_empty[PNACC];
+  uint32_t tmem_base;
+  int abort;
+  __align__(16) float rn_col[EPI_WARPS][128];
+};
+
+// grid (2 P, B) in clusters of two CTAs along x, 320 threads, dynamic smem = pair_smem<MODE>().
+// Pair p takes the 256 x 256 tiles p, p + P, ... of the pass; CTA r of the pair owns the 128-row block 2 I + r of
+// tile (I, J).  In the all-pairs pass a tile is wanted when J >= I, and of the tile (I, I) the block (2 I + 1, 2 I)
+// lies below the diagonal and is computed but not used.
+template <int MODE>
+__global__ void __launch_bounds__(THREADS, 1) k_tiles_pair(const __grid_constant__ Batch bt,
+                                                           const __grid_constant__ TmapSet tm, int kept_rows) {
+  const ImgDesc &im = bt.img[blockIdx.y];
+  TL_SCOPE(im, MODE == MODE_GRAM ? 4 : 6);
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ SharedPair sh;
+  uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_rank();
+  const bool leader = rank == 0;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < PSTAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
+    for (int a = 0; a < PNACC; ++a) { mbar_init(&sh.acc_full[a], 1); mbar_init(&sh.acc_empty[a], 2 * EPI_WARPS); }
+    sh.abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc2(&sh.tmem_base, TMEM_COLS);
+  tc_fence_before();
+  __syncthreads();
+  cluster_barrier();                                  // both CTAs' barriers exist before either is signalled
+  tc_fence_after();
+  const uint32_t tmem_base = sh.tmem_base;
+  pdl_wait();
+  pdl_trigger();
+
+  int nrows, ncols;
+  if (MODE == MODE_GRAM) { nrows = *im.q_ptr; ncols = nrows; }
+  else if (MODE == MODE_SPREAD) { nrows = im.N; ncols = im.N; }
+  else { nrows = kept_rows ? *im.q_ptr : im.N; ncols = *im.C_ptr; }
+  const int nti = (nrows + 2 * BM - 1) / (2 * BM), ntj = (ncols + PBN - 1) / PBN;
+  const int ntiles = tile_count<MODE>(nti, ntj);
+  const int P = gridDim.x >> 1, pr = blockIdx.x >> 1;
+  const int nslab = bt.d_k / BK;
+  auto wanted = [&](int I, int J) { return MODE != MODE_SPREAD || J >= I; };
+  // columns the MMA has to produce: the rows x centres pass stops at the last centre, in steps of 32
+  auto width = [&](int J) {
+    if (MODE != MODE_ASSIGN) return PBN;
+    const int left = ncols - J * PBN;
+    return left >= PBN ? PBN : ((left + 31) & ~31);
+  };
+
+  if (pr >= ntiles) {
+  } else if (warp == 0) {
+    // ---------------- TMA producer (each CTA for its own shared memory) ----------------
+    if (lane == 0) {
+      const CUtensorMap *ma = &tm.a[blockIdx.y], *mb = &tm.b[blockIdx.y];
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = pr; ok && tile < ntiles; tile += P) {
+        int I, J;
+        tile_at<MODE>(tile, nti, ntj, I, J);
+        if (!wanted(I, J)) continue;
+        const int bw = width(J);
+        for (int ks = 0; ks < nslab; ++ks, ++it) {
+          const int s = it % PSTAGES;
+          if (!mbar_wait(&sh.empty[s], ((it / PSTAGES) & 1) ^ 1)) { ok = false; break; }
+          uint8_t *a_dst = ring + (size_t)s * PSTAGE_BYTES, *b_dst = a_dst + A_BYTES;
+          if (leader) mbar_arrive_expect_tx(&sh.full[s], 2 * PSTAGE_BYTES);   // the bytes of both CTAs
+          const uint32_t bar = map_to_rank(smem_u32(&sh.full[s]), 0);
+          tma_load_2d_pair(a_dst, ma, bar, ks * BK, (2 * I + (int)rank) * BM);
+          tma_load_2d_pair(b_dst, mb, bar, ks * BK, J * PBN + (int)rank * (bw >> 1));
+        }
+      }
+      if (!ok) atomicExch(&sh.abort, 1);
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer (CTA 0 for both) ----------------
+    if (lane == 0 && leader) {
+      uint32_t it = 0, tcount = 0;
+      bool ok = true;
+      for (int tile = pr; ok && tile < ntiles; tile += P) {
+        int I, J;
+        tile_at<MODE>(tile, nti, ntj, I, J);
+        if (!wanted(I, J)) continue;
+        const uint32_t a = tcount % PNACC;
+        if (!mbar_wait(&sh.acc_empty[a], ((tcount / PNACC) & 1) ^ 1)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + a * PBN;
+        // kind::f16, fp32 accumulate, bf16 x bf16, both operands K-major, M = 256 over the pair, N = this tile's width
+        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(width(J) >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
+        for (int ks = 0; ks < nslab; ++ks, ++it) {
+          const int s = it % PSTAGES;
+          if (!mbar_wait(&sh.full[s], (it / PSTAGES) & 1)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_addr = smem_u32(ring + (size_t)s * PSTAGE_BYTES), b_addr = a_addr + A_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k)
+            umma_bf16_pair(d_tmem, smem_desc(a_addr + k * 32), smem_desc(b_addr + k * 32), idesc, (ks | k) != 0);
+          umma_commit_pair(&sh.empty[s]);          // frees the stage in both CTAs once these MMAs have read it
+        }
+        if (ok) umma_commit_pair(&sh.acc_full[a]); // accumulator complete, in both CTAs
+        ++tcount;
+      }
+      if (!ok) atomicExch(&sh.abort, 1);
+    }
+  } else {
+    // ---------------- epilogue (each CTA for its 128 rows) ----------------
+    const int ew = warp - 2;
+    const int qd = warp & 3;                        // tensor-memory lane quadrant this warp may read
+    const int half = ew >> 2;                       // which 128 columns of the tile
+    float *rn_col = sh.rn_col[ew];
+    uint32_t *tr = reinterpret_cast<uint32_t *>(ring + PRING - 1024) + ew * (32 * 36);   // all-pairs pass only
+    uint32_t tcount = 0;
+    int band = 0;
+    bool ok = true;
+    float mx = 0.f;
+    for (int tile = pr; ok && tile < ntiles; tile += P) {
+      int I, J;
+      tile_at<MODE>(tile, nti, ntj, I, J);
+      if (!wanted(I, J)) continue;
+      const uint32_t a = tcount % PNACC;
+      const int R = 2 * I + (int)rank;              // this CTA's 128-row block
+      const int cbase = J * PBN + half * 128;       // this warp's columns: one 128-column block
+      const bool skip = MODE == MODE_GRAM && cbase / BM < R;   // below the diagonal
+      const uint32_t taddr = tmem_base + a * PBN + half * 128 + ((uint32_t)(qd * 32) << 16);
+      const uint32_t rel = map_to_rank(smem_u32(&sh.acc_empty[a]), 0);
+      ok = epi_tile<MODE, 128>(im, kept_rows, R, cbase, skip, nrows, ncols, taddr, &sh.acc_full[a], (tcount / PNACC) & 1,
+                               rn_col, tr, lane, qd, band, mx, [&]() { mbar_arrive_remote(rel); });
+      if (!ok) break;
+      ++tcount;
+    }
+    if (!ok) atomicExch(&sh.abort, 1);
+    if (MODE == MODE_GRAM && band) atomicAdd(&im.cnt[PACT_CNT_BAND_DC], band);
+    if (MODE == MODE_SPREAD) {
+      const unsigned w = __reduce_max_sync(0xffffffffu, __float_as_uint(mx));
+      if (lane == 0 && w) atomicMax(reinterpret_cast<unsigned *>(&im.cnt[kCntSpread]), w);
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  cluster_barrier();                                  // nothing is in flight towards the other CTA any more
+  tc_fence_after();
+  if (warp == 1) tmem_dealloc2(tmem_base, TMEM_COLS);
   if (threadIdx.x == 0 && sh.abort) atomicMin(&im.cnt[PACT_CNT_STATUS], (int)PACT_ERR_TIMEOUT);
 }
 
@@ -507,6 +740,55 @@ constexpr int kGramBN = 128, kWideBN = 256;
 
 }  // namespace
 
+bool umma_supported(int d_k) { return g_encode != nullptr && d_k % BK == 0; }
+
+namespace {
+bool g_pair_ok = false;                               // clusters of two CTAs of the pair kernel can be launched
+
+template <int MODE>
+cudaError_t launch_pair(const Batch &bt, const TmapSet &tm, long long tiles, int kept_rows, const ClusterCfg &cfg, bool pdl,
+                        cudaStream_t st) {
+  long long P = cfg.sm_count / 2 / bt.B;              // one pair per two SMs: all pairs of the batch run at once
+  if (P > tiles) P = tiles;
+  if (P < 1) P = 1;
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3((unsigned)(2 * P), bt.B);
+  lc.blockDim = dim3(THREADS);
+  lc.dynamicSmemBytes = pair_smem<MODE>();
+  lc.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = attr;
+  lc.numAttrs = pdl ? 2 : 1;
+  return cudaLaunchKernelEx(&lc, k_tiles_pair<MODE>, bt, tm, kept_rows);
+}
+
+template <int MODE> cudaError_t pair_configure() {
+  cudaError_t e = cudaFuncSetAttribute(k_tiles_pair<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pair_smem<MODE>());
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3(2);
+  lc.blockDim = dim3(THREADS);
+  lc.dynamicSmemBytes = pair_smem<MODE>();
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  lc.attrs = attr;
+  lc.numAttrs = 1;
+  int n = 0;
+  e = cudaOccupancyMaxActiveClusters(&n, k_tiles_pair<MODE>, &lc);
+  if (e != cudaSuccess || n < 1) { (void)cudaGetLastError(); g_pair_ok = false; }
+  return cudaSuccess;
+}
+}  // namespace
+
 cudaError_t umma_configure() {
   void *fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
@@ -520,11 +802,12 @@ cudaError_t umma_configure() {
   e = cudaFuncSetAttribute(k_tiles_umma<MODE_SPREAD, kWideBN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)TileCfg<kWideBN>::SMEM);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(k_tiles_umma<MODE_ASSIGN, kWideBN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)TileCfg<kWideBN>::SMEM);
+  e = cudaFuncSetAttribute(k_tiles_umma<MODE_ASSIGN, kWideBN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)TileCfg<kWideBN>::SMEM);
+  if (e != cudaSuccess) return e;
+  g_pair_ok = true;
+  return pair_configure<MODE_SPREAD>();
 }
-
-bool umma_supported(int d_k) { return g_encode != nullptr && d_k % BK == 0; }
 
 static int umma_grid_x(long long tiles, int B, int sms) {
   long long x = sms / B;                            // one CTA per SM: all CTAs of the batch run at once
@@ -542,8 +825,7 @@ cudaError_t launch_gram_umma(const Batch &bt, int maxN, const ClusterCfg &cfg, c
   }
   const long long nb = (maxN + BM - 1) / BM;
   dim3 grid(umma_grid_x(nb * (nb + 1) / 2, bt.B, cfg.sm_count), bt.B);
-  k_tiles_umma<MODE_GRAM, kGramBN><<<grid, THREADS, TileCfg<kGramBN>::SMEM, st>>>(bt, tm, 0);
-  return cudaGetLastError();
+  return launch_k(k_tiles_umma<MODE_GRAM, kGramBN>, grid, dim3(THREADS), TileCfg<kGramBN>::SMEM, st, true, bt, tm, 0);
 }
 
 cudaError_t launch_assign_umma(const Batch &bt, int maxN, bool kept_rows, const ClusterCfg &cfg, cudaStream_t st) {
@@ -557,8 +839,7 @@ cudaError_t launch_assign_umma(const Batch &bt, int maxN, bool kept_rows, const 
   }
   const long long tiles = (long long)((maxN + BM - 1) / BM) * ((maxN + kWideBN - 1) / kWideBN);
   dim3 grid(umma_grid_x(tiles, bt.B, cfg.sm_count), bt.B);
-  k_tiles_umma<MODE_ASSIGN, kWideBN><<<grid, THREADS, TileCfg<kWideBN>::SMEM, st>>>(bt, tm, kept_rows ? 1 : 0);
-  return cudaGetLastError();
+  return launch_k(k_tiles_umma<MODE_ASSIGN, kWideBN>, grid, dim3(THREADS), TileCfg<kWideBN>::SMEM, st, true, bt, tm, kept_rows ? 1 : 0);
 }
 
 // every layer of the batch is one "image": rows and columns are all N keys of K_clu
@@ -569,10 +850,13 @@ cudaError_t launch_spread_umma(const Batch &bt, int maxN, const ClusterCfg &cfg,
     if (!encode_rows(&tm.a[b], im.Kc, im.N, im.ldKc, bt.d_k)) return cudaErrorInvalidValue;
     tm.b[b] = tm.a[b];
   }
+  if (g_pair_ok) {
+    const long long ptiles = (long long)((maxN + 2 * BM - 1) / (2 * BM)) * ((maxN + PBN - 1) / PBN);
+    return launch_pair<MODE_SPREAD>(bt, tm, ptiles, 0, cfg, false, st);
+  }
   const long long tiles = (long long)((maxN + BM - 1) / BM) * ((maxN + kWideBN - 1) / kWideBN);
   dim3 grid(umma_grid_x(tiles, bt.B, cfg.sm_count), bt.B);
-  k_tiles_umma<MODE_SPREAD, kWideBN><<<grid, THREADS, TileCfg<kWideBN>::SMEM, st>>>(bt, tm, 0);
-  return cudaGetLastError();
+  return launch_k(k_tiles_umma<MODE_SPREAD, kWideBN>, grid, dim3(THREADS), TileCfg<kWideBN>::SMEM, st, false, bt, tm, 0);
 }
 
 }  // namespace pact

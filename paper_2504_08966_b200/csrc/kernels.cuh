@@ -31,6 +31,25 @@ enum RowMode { ROWS_ALL = 0, ROWS_KEPT_LIST = 1, ROWS_PRUNED_LIST = 2 };
 constexpr int kQPartRows = 32;            // most row blocks the column sums of Q are split into
 constexpr int kHistBits = 12;             // key bits of the first-level histogram of the threshold selection
 constexpr int kHistShift = 32 - kHistBits; // a key's bin in that histogram is key >> kHistShift
+// Cooperative launch (every CTA resident at once), optionally with the programmatic-serialization attribute too.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_coop(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool pdl,
+                               Args &&...args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeCooperative;
+  attr[0].val.cooperative = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 2 : 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // Algorithm 1.  mode 0: scores, threshold, lists, survivor keys (four kernels; the first also clears what later
 // kernels accumulate into); mode 1: scores only (three kernels).
 cudaError_t launch_euti(const Batch &bt, int maxN, bool bf16, int mode, cudaStream_t st);

@@ -99,6 +99,8 @@ __global__ void __launch_bounds__(kListBlock) k_lists(const __grid_constant__ Ba
   using D = typename DistOf<T>::type;
   const ImgDesc &im = bt.img[blockIdx.y];
   TL_SCOPE(im, 8);
+  pdl_wait();
+  pdl_trigger();
   const int N = im.N;
   const int nblk = (N + kListBlock - 1) / kListBlock;
   const int b = blockIdx.x, t = threadIdx.x, lane = t & 31, w = t >> 5;
@@ -281,6 +283,8 @@ template <typename T, typename O, int VPL, int DEPTH>
 __global__ void __launch_bounds__(kMrgThreads, kMrgCtasPerSm) k_merge(const __grid_constant__ Batch bt) {
   const ImgDesc &im = bt.img[blockIdx.y];
   TL_SCOPE(im, 9);
+  pdl_wait();
+  pdl_trigger();
   const int t = threadIdx.x;
   __shared__ int4 s_rec[kMrgTile];                  // {row of H, cluster, first member position, size}
   __shared__ int s_dst[kMrgTile];                   // output row
@@ -472,13 +476,11 @@ template <typename T, bool FB>
 static cudaError_t launch_lists_t(const Batch &bt, int maxN, int spin_limit, cudaStream_t st) {
   const dim3 grid((maxN + kListBlock - 1) / kListBlock, bt.B);
   if ((long long)grid.x * grid.y <= g_lists_resident) {
-    int mode = 0;
-    void *args[] = {(void *)&bt, (void *)&mode, (void *)&spin_limit};
-    return cudaLaunchCooperativeKernel((const void *)k_lists<T, FB>, grid, dim3(kListBlock), args, 0, st);
+    return launch_coop(k_lists<T, FB>, grid, dim3(kListBlock), 0, st, true, bt, 0, spin_limit);
   }
-  k_lists<T, FB><<<grid, kListBlock, 0, st>>>(bt, 1, spin_limit);
-  k_lists<T, FB><<<grid, kListBlock, 0, st>>>(bt, 2, spin_limit);
-  return cudaGetLastError();
+  cudaError_t e = launch_k(k_lists<T, FB>, grid, dim3(kListBlock), 0, st, true, bt, 1, spin_limit);
+  if (e != cudaSuccess) return e;
+  return launch_k(k_lists<T, FB>, grid, dim3(kListBlock), 0, st, true, bt, 2, spin_limit);
 }
 
 cudaError_t launch_lists(const Batch &bt, int maxN, bool bf16, bool from_best, int spin_limit, cudaStream_t st) {
@@ -502,7 +504,7 @@ template <typename T, typename O, int VPL>
 static cudaError_t launch_merge_v(const Batch &bt, dim3 grid, cudaStream_t st) {
   constexpr int kSlotBytes = VPL * kMrgThreads * 8 * (int)sizeof(T);
   constexpr int DEPTH = kMrgRingBytes / kSlotBytes;
-  return launch_k(k_merge<T, O, VPL, DEPTH>, grid, dim3(kMrgThreads), (size_t)DEPTH * kSlotBytes, st, false, bt);
+  return launch_k(k_merge<T, O, VPL, DEPTH>, grid, dim3(kMrgThreads), (size_t)DEPTH * kSlotBytes, st, true, bt);
 }
 
 template <typename T, typename O>
