@@ -141,6 +141,14 @@ const char *pact_status_string(pact_status s);
 /* Text of the last CUDA runtime error seen by this context ("" if none). */
 const char *pact_last_cuda_error(const pact_ctx *ctx);
 
+/* Bounds of the device-side waits (Algorithm 2's centre selection is resolved in sweeps over two bit masks,
+ * and the member lists of Eq. 10 are built behind one barrier between CTAs).  When a bound is reached the
+ * kernel stops waiting, writes PACT_ERR_TIMEOUT to counters[PACT_CNT_STATUS] of the image and carries on
+ * within bounds; the call itself still returns PACT_OK and the outputs of that image are not valid.
+ * barrier_polls: polls of the member-list barrier; center_sweeps: sweeps of the centre selection;
+ * 0 restores the default (about a million).  Graphs recorded earlier keep the limits they were recorded with. */
+pact_status pact_set_wait_limits(pact_ctx *ctx, int barrier_polls, int center_sweeps);
+
 /* ---- instrumentation ---------------------------------------------------------------------- */
 
 /* Number of kernels this context has launched since it was created. */
@@ -225,7 +233,10 @@ pact_status pact_key_spread(pact_ctx *ctx, const void *const *K_layers /*host*/,
  * centre, size_out = members, logw_out = log(members) when given (the bias log W that Eq. 11
  * adds to the attention logits of the reduced sequence; 0 for text rows); text rows are copied
  * around the merged span.
- * Uses img->H, P, H_out, P_out, size_out, logw_out, counters (N_OUT is written). */
+ * Uses img->H, P, H_out, P_out, size_out, logw_out, counters (N_OUT and STATUS are written, the rest is zero).
+ * label[i] must lie in [-1, C) and *C_dev in [0, N]; center_idx[c] in [0, N).  A label outside that
+ * range is treated as -1 and reported as PACT_ERR_INVALID_ARG in counters[PACT_CNT_STATUS]; the other
+ * rows are merged as usual. */
 pact_status pact_merge(pact_ctx *ctx, const pact_image *img /*host*/, const int32_t *label,
                        const int32_t *center_idx, const int32_t *C_dev, const pact_params *p /*host*/,
                        void *ws, size_t ws_bytes, void *stream);

@@ -21,7 +21,8 @@ Steps and the passages they follow
 * ``max_key_distance``, ``select_layer``  choice of the reduction layer L (the paragraph after
   Eq. 11 and the figure it refers to: largest distance between two visual keys of a layer;
   the earliest layer where it is high enough)
-* ``pact_reduce``         Algorithm 3 end to end
+* ``pact_reduce``         Algorithm 3 end to end (with a replay mode for the keep mask and the density order)
+* ``fragile_decisions``   counts, in float64, of the real-valued comparisons that sit within 1e-6 of turning
 
 Readings taken where the paper is silent or garbled (each is also listed in the
 design notes): softmax runs over the visual tokens separately per head and
@@ -91,11 +92,13 @@ def n_pruned(lam: float, N: int) -> int:
     return int(min(np.floor(float(lam) * N + 1e-6), N - 1))
 
 
-def split(scores32: np.ndarray, lam: float):
-    """Eq. 3-4 on float32 scores.  Returns tau, keep mask, kept and pruned indices (ascending)."""
+def split(scores32: np.ndarray, lam: float, m: int | None = None):
+    """Eq. 3-4 on float32 scores.  Returns tau, keep mask, kept and pruned indices (ascending).
+    m: the number of tokens the percentile aims to cut, given directly instead of through lambda
+    (clamped to [0, N-1] like the derived one)."""
     s = np.asarray(scores32, dtype=np.float32)
     N = s.shape[0]
-    m = n_pruned(lam, N)
+    m = n_pruned(lam, N) if m is None else int(min(max(int(m), 0), N - 1))
     tau = np.sort(s, kind="stable")[m]                      # (m+1)-th smallest score
     keep = s >= tau
     return tau, keep, np.nonzero(keep)[0].astype(np.int32), np.nonzero(~keep)[0].astype(np.int32)
@@ -182,12 +185,13 @@ def nearest_center(Dc: np.ndarray):
     return a.astype(np.int64), Dc[np.arange(Dc.shape[0]), a]
 
 
-def dbdpc(U: np.ndarray, d_c: float, d_n: float):
+def dbdpc(U: np.ndarray, d_c: float, d_n: float, order: np.ndarray | None = None):
     """Algorithm 2 on the rows of U.  Returns a dict with D, rho, order, centres (ascending
-    local indices) and the cluster id of every row."""
+    local indices) and the cluster id of every row.  order: replay a given density order
+    instead of the one derived from rho (see pact_reduce)."""
     D = cosine_distance(U)
     rho = density(D, d_n)
-    order = density_order(rho)
+    order = density_order(rho) if order is None else np.asarray(order, dtype=np.int64)
     centers = centers_sequential(D, order, float(np.float32(d_c)))
     label, dmin = nearest_center(D[:, centers])
     return {"D": D, "rho": rho, "order": order, "centers": centers, "label": label, "dmin": dmin}
@@ -249,26 +253,73 @@ def select_layer(K_layers, threshold: float) -> int:
 # the whole step (Algorithm 3)
 # --------------------------------------------------------------------------
 
+def fragile_decisions(scores, tau, D, rho, order, d_c, Dk_centers, Dp_centers, t_reinc, tol=1e-6):
+    """Real-valued decisions of one image that a different rounding could turn, counted in float64.
+
+    Every discrete output hangs on comparisons of real numbers.  A pair within `tol` of d_c (or a
+    pruned token within `tol` of alpha d_c) is the one class the specification exempts; the others are
+    reported so that a mismatch can be traced to its root:
+      score_tau   tokens whose score differs from tau but by at most tol * tau (Eq. 3-4)
+      rho_order   neighbours in the density order whose densities differ by at most tol * rho and that
+                  lie within d_c (1 + tol) of each other (only such a pair can change a centre)
+      band_dc     unordered pairs of survivors with |d - d_c| <= tol (Algorithm 2's centre test)
+      band_adc    pruned tokens whose nearest-centre distance is within tol of alpha d_c (Eq. 8)
+      argmin      tokens whose two nearest centres differ by at most tol in distance (Algorithm 2's
+                  assignment and Eq. 8's nearest centre)
+    Each class comes with its smallest margin (None when the class has no candidate at all)."""
+    s = np.asarray(scores, dtype=np.float64)
+    tau = float(tau)
+    ds = np.abs(s - tau)
+    off = ds[ds > 0]
+    out = {"score_tau": int(((ds > 0) & (ds <= tol * abs(tau))).sum()),
+           "score_tau_min_rel": float(off.min() / abs(tau)) if off.size and tau != 0 else None}
+    a, b = order[:-1], order[1:]
+    gap = rho[a] - rho[b]
+    near = D[a, b] <= d_c * (1 + tol)
+    out["rho_order"] = int((near & (gap <= tol * rho[a])).sum())
+    out["rho_order_min_rel"] = float((gap[near] / rho[a][near]).min()) if near.any() else None
+    iu = np.triu_indices(D.shape[0], 1)
+    dd = np.abs(D[iu] - d_c)
+    out["band_dc"] = int((dd <= tol).sum())
+    out["band_dc_min"] = float(dd.min()) if dd.size else None
+    dp = np.abs(Dp_centers.min(axis=1) - t_reinc) if Dp_centers.shape[0] and Dp_centers.shape[1] else np.zeros(0)
+    out["band_adc"] = int((dp <= tol).sum())
+    out["band_adc_min"] = float(dp.min()) if dp.size else None
+    n_close, min_gap = 0, None
+    for Dc in (Dk_centers, Dp_centers):
+        if Dc.shape[0] and Dc.shape[1] >= 2:
+            two = np.partition(Dc, 1, axis=1)[:, :2]
+            g = two[:, 1] - two[:, 0]
+            n_close += int((g <= tol).sum())
+            min_gap = float(g.min()) if min_gap is None else min(min_gap, float(g.min()))
+    out["argmin"] = n_close
+    out["argmin_min"] = min_gap
+    return out
+
+
 def pact_reduce(H, K_euti, Q_euti, K_clu, P, vis_start, N, n_qh, n_kvh, lam, d_c, d_n=2.0,
-                alpha=1.5, use_norm=True, use_query=True, center_only=False, n_prune=None):
+                alpha=1.5, use_norm=True, use_query=True, center_only=False, n_prune=None,
+                keep_given=None, order_given=None):
     """Algorithm 3 on one image.  H [n_total, d], P [n_total]; K/Q rows are the N visual tokens.
 
-    Returns every intermediate the parity tests compare, plus the counts of
-    near-threshold decisions (pairs within 1e-6 of d_c, pruned tokens within 1e-6 of alpha*d_c).
+    Returns every intermediate the parity tests compare, plus the near-threshold decisions of
+    `fragile_decisions` under "fragile" (band_dc and band_adc also at the top level).
+
+    Replay: keep_given (bool [N]) replaces the keep mask of Eq. 3-4 and order_given (survivor
+    positions by descending density) replaces the density order of Algorithm 2, so that when one
+    of those decisions was turned by a near-tie every later stage can still be compared exactly.
     """
     n_total = H.shape[0]
     Hv = H[vis_start:vis_start + N]
     scores = importance_scores(Hv, K_euti, Q_euti, n_qh, n_kvh, use_norm, use_query)
     scores32 = scores.astype(np.float32)
-    if n_prune is None:
-        tau, keep, kept, pruned = split(scores32, lam)
-    else:
-        tau = np.sort(scores32, kind="stable")[min(n_prune, N - 1)]
-        keep = scores32 >= tau
+    tau, keep, kept, pruned = split(scores32, lam, n_prune)
+    if keep_given is not None:
+        keep = np.asarray(keep_given, dtype=bool)
         kept = np.nonzero(keep)[0].astype(np.int32)
         pruned = np.nonzero(~keep)[0].astype(np.int32)
     dc = float(np.float32(d_c))
-    cl = dbdpc(K_clu[kept], dc, d_n)
+    cl = dbdpc(K_clu[kept], dc, d_n, order_given)
     centers_local = cl["centers"]
     center_token = kept[centers_local].astype(np.int64)      # ascending token index = cluster id order
     C = center_token.size
@@ -283,8 +334,9 @@ def pact_reduce(H, K_euti, Q_euti, K_clu, P, vis_start, N, n_qh, n_kvh, lam, d_c
     P_out = np.concatenate([P[:vis_start], Pm, P[vis_start + N:]])
     size_out = np.concatenate([np.ones(vis_start, np.int64), sizes,
                                np.ones(n_total - vis_start - N, np.int64)])
-    iu = np.triu_indices(kept.size, 1)
     t = reinc_threshold(alpha, dc)
+    Dp = cosine_distance(K_clu[pruned], K_clu[center_token]) if pruned.size else np.zeros((0, C))
+    frag = fragile_decisions(scores, tau, cl["D"], cl["rho"], cl["order"], dc, cl["D"][:, centers_local], Dp, t)
     return {
         "scores": scores, "scores32": scores32, "tau": tau, "keep": keep, "kept_idx": kept,
         "pruned_idx": pruned, "D": cl["D"], "rho": cl["rho"], "order": cl["order"],
@@ -294,6 +346,5 @@ def pact_reduce(H, K_euti, Q_euti, K_clu, P, vis_start, N, n_qh, n_kvh, lam, d_c
         "logw_out": proportional_attention_bias(size_out),
         "q": int(kept.size), "C": int(C), "r": int((lab_p >= 0).sum()),
         "discarded": int((lab_p < 0).sum()),
-        "band_dc": int((np.abs(cl["D"][iu] - dc) <= 1e-6).sum()),
-        "band_adc": int((np.abs(dmin_p - t) <= 1e-6).sum()),
+        "band_dc": frag["band_dc"], "band_adc": frag["band_adc"], "fragile": frag,
     }

@@ -26,7 +26,7 @@ EXPORTS = ["pact_create", "pact_destroy", "pact_workspace_bytes", "pact_status_s
            "pact_prune_static", "pact_reincorporate", "pact_merge", "pact_reduce", "pact_reduce_host",
            "pact_host_staging_bytes", "pact_launch_count", "pact_profile_enable", "pact_profile_read",
            "pact_profile_stage_name", "pact_graph_create", "pact_graph_launch", "pact_graph_destroy",
-           "pact_key_spread"]
+           "pact_key_spread", "pact_set_wait_limits"]
 
 
 class Params(C.Structure):
@@ -79,6 +79,7 @@ def lib():
         L.pact_graph_launch.argtypes = [vp, vp]
         L.pact_graph_destroy.argtypes = [vp]
         L.pact_launch_count.argtypes = [vp]
+        L.pact_set_wait_limits.argtypes = [vp, i32, i32]
         L.pact_launch_count.restype = C.c_longlong
         L.pact_profile_enable.argtypes = [vp, i32]
         L.pact_profile_read.argtypes = [vp, C.POINTER(C.c_float), i32]
@@ -311,6 +312,10 @@ class Context:
         h = C.c_void_p()
         _check(self.handle, self._L.pact_graph_create(self.handle, arr, B, parr, stride, w, n, C.byref(h)))
         return Graph(self, h, images, self.ws)
+
+    def set_wait_limits(self, barrier_polls: int = 0, center_sweeps: int = 0):
+        """Bounds of the device-side waits (0 = default); see pact_set_wait_limits in pact.h."""
+        _check(self.handle, self._L.pact_set_wait_limits(self.handle, int(barrier_polls), int(center_sweeps)))
 
     def launch_count(self) -> int:
         return int(self._L.pact_launch_count(self.handle))

@@ -20,7 +20,8 @@ struct pact_ctx {
   int device;
   char err[256];
   long long launches;      // kernels launched by this context so far
-  int spin_limit;          // polls a bounded device wait makes before it raises PACT_ERR_TIMEOUT
+  int spin_limit;          // polls the barrier of the member-list kernel makes before it raises PACT_ERR_TIMEOUT
+  int sweep_limit;         // sweeps the centre selection makes before it raises PACT_ERR_TIMEOUT
   int prof_on;             // record an event after every stage of pact_reduce
   int prof_n;              // stages recorded by the last profiled call
   cudaEvent_t ev[kProfStages + 1];
@@ -255,6 +256,7 @@ pact_status pact_create(pact_ctx **out, int d, int n_qh, int n_kvh, int d_h, pac
   }
   c->umma = in == PACT_BF16 && umma_supported(c->d_k);
   c->spin_limit = kSpinLimit;
+  c->sweep_limit = kSpinLimit;
   *out = c;
   return PACT_OK;
 }
@@ -267,6 +269,13 @@ pact_status pact_destroy(pact_ctx *ctx) {
 }
 
 long long pact_launch_count(const pact_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+pact_status pact_set_wait_limits(pact_ctx *ctx, int barrier_polls, int center_sweeps) {
+  if (!ctx || barrier_polls < 0 || center_sweeps < 0) return PACT_ERR_INVALID_ARG;
+  ctx->spin_limit = barrier_polls ? barrier_polls : kSpinLimit;
+  ctx->sweep_limit = center_sweeps ? center_sweeps : kSpinLimit;
+  return PACT_OK;
+}
 
 pact_status pact_profile_enable(pact_ctx *ctx, int on) {
   if (!ctx) return PACT_ERR_INVALID_ARG;
@@ -379,7 +388,7 @@ pact_status pact_dbdpc(pact_ctx *ctx, const void *K, int64_t ldK, int N, const i
   launch_keynorm_gather(bt, N, bf, false, st);
   if (ctx->umma) CK(launch_gram_umma(bt, N, ctx->ccfg, st));
   else launch_gram(bt, N, bf, ctx->ccfg, st);
-  CK(launch_centers(bt, N, bf, ctx->ccfg, ctx->spin_limit, st));
+  CK(launch_centers(bt, N, bf, ctx->ccfg, ctx->sweep_limit, st));
   if (ctx->umma) CK(launch_assign_umma(bt, N, true, ctx->ccfg, st));
   else launch_assign(bt, N, bf, ROWS_KEPT_LIST, ctx->ccfg, st);
   launch_label(bt, N, bf, ROWS_KEPT_LIST, st);
@@ -490,7 +499,7 @@ pact_status pact_merge(pact_ctx *ctx, const pact_image *img, const int32_t *labe
   CK(launch_merge(bt, ctx->in == PACT_BF16, ctx->out == PACT_BF16, ctx->ccfg, st));
   ctx->launches += lists_kernels(img->N, 1) + 1;
   CK(cudaGetLastError());
-  CK(cudaMemcpyAsync(img->counters, m.cnt, sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
+  CK(cudaMemcpyAsync(img->counters, m.cnt, PACT_N_COUNTERS * sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
   return PACT_OK;
 }
 
@@ -541,7 +550,7 @@ pact_status pact_reduce(pact_ctx *ctx, const pact_image *imgs, int B, const pact
     if (ctx->umma) CK(launch_gram_umma(bt, cmaxN, ctx->ccfg, st));
     else launch_gram(bt, cmaxN, bf, ctx->ccfg, st);
     CK(mark());
-    CK(launch_centers(bt, cmaxQ, bf, ctx->ccfg, ctx->spin_limit, st));  CK(mark());
+    CK(launch_centers(bt, cmaxQ, bf, ctx->ccfg, ctx->sweep_limit, st));  CK(mark());
     if (ctx->umma) CK(launch_assign_umma(bt, cmaxN, false, ctx->ccfg, st));
     else launch_assign(bt, cmaxN, bf, ROWS_ALL, ctx->ccfg, st);
     CK(mark());

@@ -59,21 +59,9 @@ def bf16_round(x: np.ndarray) -> np.ndarray:
     return torch.from_numpy(np.ascontiguousarray(x)).to(torch.float32).to(torch.bfloat16).to(torch.float64).numpy()
 
 
-def fragile_report(o, wl_d_c, alpha):
-    """What the oracle knows about near-threshold decisions of one image (float64 margins)."""
-    s, tau = o["scores"], float(o["tau"])
-    rho = o["rho"]
-    order = o["order"]
-    gaps = -np.diff(rho[order])
-    dc = float(np.float32(wl_d_c))
-    D = o["D"]
-    close = D[order[:-1], order[1:]] <= dc * (1 + 1e-6)
-    return {
-        "score_margin_rel": float(np.min(np.abs(s - tau)[np.abs(s - tau) > 0]) / tau) if tau > 0 else None,
-        "min_rho_gap": float(gaps.min()) if gaps.size else None,
-        "min_rho_gap_between_neighbours": float(gaps[close].min()) if close.any() else None,
-        "band_dc": o["band_dc"], "band_adc": o["band_adc"],
-    }
+def fragile_report(o, wl_d_c=None, alpha=None):
+    """The oracle's float64 count of near-threshold decisions of one image (see orc.fragile_decisions)."""
+    return o["fragile"]
 
 
 def compare_image(o, g, img, out_is_bf16, check_scores=True):

@@ -213,7 +213,10 @@ def test_strided_inputs():
     n_out = int(im.counters[0])
     assert n_out == o["n_out"] and np.array_equal(im.label.cpu().numpy(), o["label"])
     got = im.H_out[:n_out].double().cpu().numpy()
-    assert np.abs(got - o["H_out"]).max() <= 2e-3 * np.abs(o["H_out"]).max()
+    num = np.abs(got - o["H_out"]).max(axis=1)
+    den = np.maximum(np.abs(o["H_out"]).max(axis=1), 1e-300)
+    assert (num / den).max() <= 2e-3                        # per row, as everywhere else
+    assert np.array_equal(im.P_out[:n_out].cpu().numpy(), o["P_out"])
 
 
 def test_bitwise_deterministic_run_to_run():
@@ -398,7 +401,14 @@ def test_stage_dbdpc_reincorporate_merge(stage_case):
     assert np.array_equal(label.cpu().numpy(), want)
     rel = np.abs(rho[:o["q"]].cpu().numpy() - o["rho"]) / o["rho"]
     assert rel.max() < 1e-6
-    assert np.array_equal(np.argsort(-rho[:o["q"]].cpu().numpy().astype(np.float64), kind="stable")[:50], o["order"][:50]) or True
+    # the float32 densities the stage returns give the oracle's order wherever the oracle's own densities are
+    # further apart than float32 resolves: compare the order up to runs of such near-equal neighbours
+    got_rho = rho[:o["q"]].cpu().numpy().astype(np.float64)
+    ord_o = o["order"]
+    gaps = o["rho"][ord_o[:-1]] - o["rho"][ord_o[1:]]
+    clear = gaps > 4e-7 * o["rho"][ord_o[:-1]]             # float32 keeps these apart (ulp 6e-8, error <= 1e-6 checked above)
+    assert clear.mean() > 0.5
+    assert np.all(got_rho[ord_o[:-1]][clear] >= got_rho[ord_o[1:]][clear])
     # reincorporation from the oracle's centres
     pruned = torch.from_numpy(o["pruned_idx"]).cuda()
     m_dev = torch.tensor([o["pruned_idx"].size], dtype=torch.int32, device="cuda")
@@ -538,3 +548,76 @@ def test_invalid_arguments_are_rejected_before_launch():
     with pytest.raises(pb.PactError):
         pb.Context(100, 4, 3, 16)                   # n_qh not a multiple of n_kvh
     torch.cuda.synchronize()
+
+
+# ------------------------------------------------------------------ given number of pruned tokens, wait limits, bad labels
+
+@pytest.mark.parametrize("m", [0, 1, 333, 699, 5000])
+def test_given_number_of_pruned_tokens(m):
+    """pact_params.n_prune replaces the m derived from lambda (Eq. 3-4 with a given m)."""
+    from paper_2504_08966_b200 import binding as pb
+    wl = _small(seed=83)
+    params = pb.make_params(lam=0.9, d_c=wl.d_c, d_n=wl.d_n, alpha=wl.alpha, n_prune=m)
+    outs, _ = gpu_reduce(wl, torch.float32, params=params)
+    o = oracle_image(wl, wl.images[0], n_prune=m)
+    bad = compare_image(o, outs[0], wl.images[0], False)
+    assert not bad, f"n_prune={m}: {bad}; fragile: {o['fragile']}"
+    assert outs[0]["counters"][9] <= min(m, wl.images[0].N - 1)      # pruned tokens, ties at tau are kept
+
+
+def test_centre_sweep_limit_is_reported_and_the_context_recovers():
+    """A wait that runs out must surface as PACT_ERR_TIMEOUT in the image's status word, with the call
+    returning normally, and must leave the context usable: one sweep is not enough for an image whose
+    centres depend on one another; the default limit then gives the oracle's result again."""
+    from paper_2504_08966_b200 import binding as pb
+    wl = workloads.single_image(seed=29, N=2000, T=8, n_blobs=50)
+    img = wl.images[0]
+    ctx = pb.Context(wl.d, wl.n_qh, wl.n_kvh, wl.d_h, wl.dtype, torch.bfloat16)
+    params = pb.make_params(lam=wl.lam, d_c=wl.d_c, d_n=wl.d_n, alpha=wl.alpha)
+    im = pb.device_image(img, torch.bfloat16)
+    ctx.pact_reduce([im], params)
+    torch.cuda.synchronize()
+    assert int(im.counters[pb.CNT["status"]]) == 0 and int(im.counters[pb.CNT["sweeps"]]) >= 2
+    good = im.label.clone()
+    ctx.set_wait_limits(center_sweeps=1)
+    ctx.pact_reduce([im], params)                           # returns normally
+    torch.cuda.synchronize()
+    assert int(im.counters[pb.CNT["status"]]) == -5         # PACT_ERR_TIMEOUT
+    n_out = int(im.counters[pb.CNT["n_out"]])
+    assert 0 <= n_out <= img.H.shape[0]
+    ctx.set_wait_limits()                                   # defaults
+    ctx.pact_reduce([im], params)
+    torch.cuda.synchronize()
+    assert int(im.counters[pb.CNT["status"]]) == 0
+    assert torch.equal(im.label, good)
+    o = oracle_image(wl, img)
+    assert np.array_equal(im.label.cpu().numpy(), o["label"])
+
+
+def test_merge_reports_a_label_outside_its_range(stage_case):
+    """pact_merge takes labels from the caller: one that names no cluster is dropped and reported, the other
+    rows are merged as usual and nothing is written out of bounds."""
+    wl, img, o, ctx, im, params = stage_case
+    label = o["label"].astype(np.int32).copy()
+    victim = int(np.nonzero(label >= 0)[0][5])
+    label[victim] = o["C"]                                  # one past the last cluster id
+    lab_d = torch.from_numpy(label).cuda()
+    cidx = torch.from_numpy(o["center_idx"].astype(np.int32)).cuda()
+    C_dev = torch.tensor([o["C"]], dtype=torch.int32, device="cuda")
+    im.H_out.zero_()
+    ctx.pact_merge(im, lab_d, cidx, C_dev, params)
+    torch.cuda.synchronize()
+    assert int(im.counters[pb_status()]) == -1              # PACT_ERR_INVALID_ARG
+    lab_ref = o["label"].copy()
+    lab_ref[victim] = -1
+    Hm, Pm, sizes = orc.merge(f64(img.H)[img.vis_start:img.vis_start + img.N], lab_ref, o["C"], o["center_idx"],
+                              img.P.numpy()[img.vis_start:img.vis_start + img.N])
+    got = im.H_out[img.vis_start:img.vis_start + o["C"]].double().cpu().numpy()
+    num = np.abs(got - Hm).max(axis=1)
+    assert (num / np.maximum(np.abs(Hm).max(axis=1), 1e-300)).max() <= 2e-3
+    assert np.array_equal(im.size_out[img.vis_start:img.vis_start + o["C"]].cpu().numpy(), sizes)
+
+
+def pb_status():
+    from paper_2504_08966_b200 import binding as pb
+    return pb.CNT["status"]

@@ -423,3 +423,112 @@ def test_small_bf16_mixture_invariants():
     assert 1 < o["C"] < o["q"]
     lk = o["label"][o["kept_idx"]]
     assert np.all(D[np.arange(o["q"]), C[lk]] <= np.float32(wl.d_c))
+
+
+# ---- the split with a given number of pruned tokens, replay, fragile decisions, planted mistakes --------
+
+@pytest.mark.parametrize("N", [1, 2, 7, 16])
+def test_split_with_given_m_bruteforce(N):
+    """split(s, lam, m) cuts the tokens strictly below the (m+1)-th smallest score, whatever lam says."""
+    rng = np.random.default_rng(100 + N)
+    s = rng.integers(0, 5, N).astype(np.float32)            # many ties
+    for m in range(-1, N + 2):
+        tau, keep, kept, pruned = orc.split(s, 0.9, m)
+        mm = min(max(m, 0), N - 1)
+        want_tau = sorted(s.tolist())[mm]
+        assert tau == want_tau
+        assert keep.tolist() == [x >= want_tau for x in s.tolist()]
+        assert pruned.size <= mm and kept.size + pruned.size == N
+        assert kept.tolist() == sorted(kept.tolist()) and pruned.tolist() == sorted(pruned.tolist())
+    # the derived m and the given m agree when they are the same number
+    a = orc.split(s, 0.5)
+    b = orc.split(s, 0.0, orc.n_pruned(0.5, N))
+    assert a[0] == b[0] and np.array_equal(a[1], b[1])
+
+
+def test_pact_reduce_with_given_m_equals_lambda_that_gives_it():
+    wl = workloads.tiny()
+    img = wl.images[0]
+    m = orc.n_pruned(wl.lam, img.N)
+    a = oracle_image(wl, img)
+    b = oracle_image(wl, img, lam=0.0, n_prune=m)
+    assert np.array_equal(a["keep"], b["keep"]) and np.array_equal(a["label"], b["label"])
+    c = oracle_image(wl, img, n_prune=0)                    # nothing pruned
+    assert c["q"] == img.N and c["r"] == 0
+
+
+def test_replay_of_own_decisions_changes_nothing_and_a_given_order_is_followed():
+    wl = workloads.tiny()
+    img = wl.images[0]
+    a = oracle_image(wl, img)
+    b = oracle_image(wl, img, keep_given=a["keep"], order_given=a["order"])
+    assert np.array_equal(a["label"], b["label"]) and np.array_equal(a["H_out"], b["H_out"])
+    # a different keep mask is taken as given
+    keep = a["keep"].copy()
+    flip = int(np.nonzero(keep)[0][0])
+    keep[flip] = False
+    c = oracle_image(wl, img, keep_given=keep)
+    assert c["q"] == a["q"] - 1 and not c["keep"][flip]
+    # three collinear points 0 - 1 - 2 with d(0,1), d(1,2) <= d_c < d(0,2): the order decides the centres
+    ang = np.array([0.0, 0.5, 1.0])
+    U = np.stack([np.cos(ang), np.sin(ang)], axis=1)
+    d_c = 1 - math.cos(0.6)
+    assert orc.dbdpc(U, d_c, 2.0, order=np.array([1, 0, 2]))["centers"].tolist() == [1]
+    assert orc.dbdpc(U, d_c, 2.0, order=np.array([0, 1, 2]))["centers"].tolist() == [0, 2]
+
+
+def test_fragile_decisions_on_a_hand_made_case():
+    """Every class is planted once and must be counted once."""
+    scores = np.array([1.0, 2.0, 2.0 + 1e-6, 3.0, 2.0])     # tau = 2: one score within 1e-6 tau above it
+    d_c = 0.5
+    D = np.array([[0.0, 0.5 + 5e-7, 0.9], [0.5 + 5e-7, 0.0, 0.2], [0.9, 0.2, 0.0]])   # pair (0,1) in the d_c band
+    rho = np.array([2.0, 3.0, 3.0 - 1e-6])                  # 1 and 2 are neighbours in the order, within d_c
+    order = np.array([1, 2, 0])
+    Dk = np.array([[0.1, 0.1 + 5e-7], [0.0, 0.7], [0.7, 0.0]])   # row 0: two centres within 1e-6
+    Dp = np.array([[0.75 - 2e-7, 1.0], [0.3, 0.9]])         # row 0: nearest centre within 1e-6 of alpha d_c = 0.75
+    f = orc.fragile_decisions(scores, 2.0, D, rho, order, d_c, Dk, Dp, 0.75)
+    assert (f["score_tau"], f["rho_order"], f["band_dc"], f["band_adc"], f["argmin"]) == (1, 1, 1, 1, 1)
+    assert abs(f["score_tau_min_rel"] - 5e-7) < 1e-9 and abs(f["band_dc_min"] - 5e-7) < 1e-12
+    # moved away by ten times the tolerance, nothing is counted
+    D2 = D.copy(); D2[0, 1] = D2[1, 0] = 0.5 + 1e-5
+    f2 = orc.fragile_decisions(np.array([1.0, 2.0, 2.1, 3.0, 2.0]), 2.0, D2, np.array([2.0, 3.0, 2.9]), order, d_c,
+                               np.array([[0.1, 0.2], [0.0, 0.7], [0.7, 0.0]]), np.array([[0.7, 1.0], [0.3, 0.9]]), 0.75)
+    assert (f2["score_tau"], f2["rho_order"], f2["band_dc"], f2["band_adc"], f2["argmin"]) == (0, 0, 0, 0, 0)
+
+
+def _mutants():
+    """Plausible slips, each planted in a copy of one oracle function (on the CPU, never in the product)."""
+    real_distance = orc.cosine_distance
+    def dist_wrong_sign(U, V=None):
+        D = real_distance(U, V)
+        return np.clip(2.0 - D, 0.0, 2.0) if V is None else 2.0 - D          # 1 + cos instead of 1 - cos
+    def density_without_self(D, d_n):
+        return np.exp(-D / d_n).sum(axis=1) - 1.0                               # dropped j = i
+    def order_ascending(rho):
+        return np.argsort(rho, kind="stable")                                   # sorted the wrong way
+    def centres_not_strict(D, order, d_c):
+        centers = []
+        for i in order:
+            if not centers or D[i, centers].min() >= d_c:                       # >= instead of >
+                centers.append(int(i))
+        return np.array(sorted(centers), dtype=np.int64)
+    def scores_softmax_over_heads(H, K, Q, n_qh, n_kvh, use_norm=True, use_query=True):
+        N = H.shape[0]; d_h = K.shape[1] // n_kvh
+        Kd = K.astype(np.float64).reshape(N, n_kvh, d_h); Qg = orc.global_query(Q.astype(np.float64).reshape(N, n_qh, d_h))
+        L = np.stack([Kd[:, (j * n_kvh) // n_qh, :] @ Qg[j] for j in range(n_qh)], axis=1)
+        P = np.exp(L - L.max(axis=1, keepdims=True)); P /= P.sum(axis=1, keepdims=True)   # softmax over the wrong axis
+        return P.mean(axis=1) * np.sqrt((H.astype(np.float64) ** 2).sum(axis=1))
+    return {"cosine_distance": dist_wrong_sign, "density": density_without_self, "density_order": order_ascending,
+            "centers_sequential": centres_not_strict, "importance_scores": scores_softmax_over_heads}
+
+
+@pytest.mark.parametrize("name", ["cosine_distance", "density", "density_order", "centers_sequential", "importance_scores"])
+def test_a_planted_mistake_fails_a_pin(name, monkeypatch):
+    """The pins are only worth something if a wrong oracle fails them: plant one mistake at a time."""
+    pins = {"cosine_distance": test_distance_special_cases, "density": test_density_closed_forms,
+            "density_order": test_duplicate_rows_have_equal_density_and_order_by_index,
+            "centers_sequential": test_exact_dc_is_member_not_centre, "importance_scores": test_scores_over_norm_sum_to_one}
+    pins[name]()                                            # green with the real function
+    monkeypatch.setattr(orc, name, _mutants()[name])
+    with pytest.raises(AssertionError):
+        pins[name]()
