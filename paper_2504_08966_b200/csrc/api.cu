@@ -95,6 +95,7 @@ size_t carve_image(const pact_ctx *c, int N, char *base, ImgDesc *im) {
   cv.take(m.members, (size_t)N * sizeof(int4));
   cv.take(m.csize, (size_t)Np * sizeof(int32_t));
   cv.take(m.cticket, (size_t)Np * sizeof(int32_t));
+  cv.take(m.rtick, (size_t)Wp * sizeof(int32_t));
   // two partial sums per CTA of k_merge (a range boundary cuts at most two clusters)
   cv.take(m.mpart, (size_t)2 * merge_ctas(c->ccfg.sm_count, 1) * c->d * sizeof(float));
   return cv.off;
@@ -460,8 +461,17 @@ pact_status pact_reincorporate(pact_ctx *ctx, const void *K, int64_t ldK, int N,
   m.m_ptr = m_dev; m.C_ptr = C_dev; m.cidx_ptr = center_idx;
   m.label = label;                      // updated in place
   CK(cudaMemsetAsync(m.cnt, 0, (kCntInts + kTickInts) * sizeof(int32_t), st));
-  launch_center_key_gather(bt, N, bf, st);
-  launch_assign(bt, N, bf, ROWS_PRUNED_LIST, ctx->ccfg, st);
+  if (ctx->umma) {
+    // the rows x centres pass on the tensor cores covers every token (the survivors' distances are computed
+    // and not used), so every token needs its inverse key norm
+    launch_key_rnorm(bt, N, bf, st);
+    launch_center_key_gather(bt, N, bf, st);
+    CK(launch_assign_umma(bt, N, false, ctx->ccfg, st));
+    ctx->launches += 1;
+  } else {
+    launch_center_key_gather(bt, N, bf, st);
+    launch_assign(bt, N, bf, ROWS_PRUNED_LIST, ctx->ccfg, st);
+  }
   launch_label(bt, N, bf, ROWS_PRUNED_LIST, st);
   ctx->launches += 3;
   CK(cudaGetLastError());
@@ -551,12 +561,16 @@ pact_status pact_reduce(pact_ctx *ctx, const pact_image *imgs, int B, const pact
     else launch_gram(bt, cmaxN, bf, ctx->ccfg, st);
     CK(mark());
     CK(launch_centers(bt, cmaxQ, bf, ctx->ccfg, ctx->sweep_limit, st));  CK(mark());
-    if (ctx->umma) CK(launch_assign_umma(bt, cmaxN, false, ctx->ccfg, st));
+    // on the tensor-core path the labels and member counts are formed as the rows x centres pass finishes
+    // groups of rows, and one kernel places the members; otherwise k_lists does both
+    if (ctx->umma) CK(launch_assign_umma(bt, cmaxN, false, ctx->ccfg, st, true));
     else launch_assign(bt, cmaxN, bf, ROWS_ALL, ctx->ccfg, st);
     CK(mark());
-    CK(launch_lists(bt, cmaxN, bf, true, ctx->spin_limit, st));  CK(mark());
+    if (ctx->umma) CK(launch_members(bt, cmaxN, st));
+    else CK(launch_lists(bt, cmaxN, bf, true, ctx->spin_limit, st));
+    CK(mark());
     CK(launch_merge(bt, bf, ctx->out == PACT_BF16, ctx->ccfg, st));  CK(mark());
-    ctx->launches += euti_kernels(0) + 4 + lists_kernels(cmaxN, nb);
+    ctx->launches += euti_kernels(0) + 4 + (ctx->umma ? 1 : lists_kernels(cmaxN, nb));
     CK(cudaGetLastError());
     for (int b = 0; b < nb; ++b)
       CK(cudaMemcpyAsync(bt.img[b].counters_user, bt.img[b].cnt, PACT_N_COUNTERS * sizeof(int32_t),

@@ -7,7 +7,7 @@
 #include <cooperative_groups.h>
 
 #include "kernels.cuh"
-#ifdef PACT_TL_EUTI
+#if defined(PACT_TL_EUTI) || defined(PACT_TL_MERGE)
 #undef TL_POINT
 #define TL_POINT(im, kid)
 #endif

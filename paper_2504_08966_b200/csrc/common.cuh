@@ -70,6 +70,7 @@ struct ImgDesc {
   int4 *members;         // [N] {token, cluster, first member position of the cluster, cluster size}, cluster order
   int32_t *csize;        // [Np] members of cluster c
   int32_t *cticket;      // [Np] chunks of cluster c that are finished
+  int32_t *rtick;        // [Wp] epilogue warps of the rows x centres pass that are done with a group of 32 tokens
   float *mpart;          // [2 * merge CTAs][d] sums of the clusters that a range boundary of k_merge cuts
   int32_t *tick;         // [kTickInts] tickets of k_qsum, one per column group; zero when a call starts (cleared with cnt)
   int32_t *cnt;          // [PACT_N_COUNTERS] + [16] ticket of the global query, [19] barrier of k_lists, [20] members of all clusters

@@ -52,7 +52,7 @@ __global__ void __launch_bounds__(kQsumThreads, 4) k_qsum(const __grid_constant_
   if (do_init) {
     const int gt = blockIdx.x * kQsumThreads + t, gs = gridDim.x * kQsumThreads;
     for (int r = gt; r < im.Np; r += gs) { im.rho_fix[r] = 0ull; im.csize[r] = 0; im.cticket[r] = 0; }
-    for (int wd = gt; wd < im.Wp; wd += gs) { im.cmask[wd] = 0u; im.rmask[wd] = 0u; }
+    for (int wd = gt; wd < im.Wp; wd += gs) { im.cmask[wd] = 0u; im.rmask[wd] = 0u; im.rtick[wd] = 0; }
     for (int i = gt; i < N; i += gs) im.best[i] = kBestInit;
     uint4 *tab = reinterpret_cast<uint4 *>(im.cnt_cb);
     const int nq = im.Np * (im.nbp / 8);
@@ -727,7 +727,7 @@ __global__ void __launch_bounds__(1024) k_select_gather(const __grid_constant__ 
   if (do_gather) {   // per-call initialisation, spread over the grid
     const int gt = blockIdx.x * 1024 + t, gs = gridDim.x * 1024;
     for (int r = gt; r < im.Np; r += gs) { im.rho_fix[r] = 0ull; im.csize[r] = 0; im.cticket[r] = 0; }
-    for (int wd = gt; wd < im.Wp; wd += gs) { im.cmask[wd] = 0u; im.rmask[wd] = 0u; }
+    for (int wd = gt; wd < im.Wp; wd += gs) { im.cmask[wd] = 0u; im.rmask[wd] = 0u; im.rtick[wd] = 0; }
     for (int i = gt; i < N; i += gs) im.best[i] = kBestInit;
     uint4 *tab = reinterpret_cast<uint4 *>(im.cnt_cb);
     const int nq = im.Np * (im.nbp / 8);

@@ -30,7 +30,10 @@ constexpr int BK = 64;            // bf16 elements per K-slab = one 128-byte swi
 constexpr int A_BYTES = BM * BK * 2;
 constexpr int TMEM_COLS = 512;    // all of an SM's tensor memory
 constexpr int MAX_STAGES = 6;
-constexpr int EPI_WARPS = 8;      // per tensor-memory lane quadrant EPI_WARPS / 4 warps share the columns
+#ifndef PACT_EPI_WARPS
+#define PACT_EPI_WARPS 8
+#endif
+constexpr int EPI_WARPS = PACT_EPI_WARPS;      // per tensor-memory lane quadrant EPI_WARPS / 4 warps share the columns
                                   // (16 measured the same on the all-pairs pass and slower on the others)
 constexpr int THREADS = 64 + EPI_WARPS * 32;
 constexpr int MAX_ACC = 4;
@@ -40,7 +43,7 @@ constexpr int MAX_ACC = 4;
 template <int BN> struct TileCfg {
   static constexpr int B_BYTES = BN * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int STAGES = BN == 256 ? 4 : 5;
+  static constexpr int STAGES = (BN == 256 || EPI_WARPS > 8) ? 4 : 5;
   static constexpr int NACC = TMEM_COLS / BN;      // accumulators in tensor memory
   static constexpr int HALF = BN / (EPI_WARPS / 4); // columns per epilogue warp
   // BN = 128 (all-pairs pass): one 32 x 32 exchange buffer per epilogue warp behind the ring
@@ -105,6 +108,7 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
 
 struct Shared {
   uint64_t full[MAX_STAGES], empty[MAX_STAGES], acc_full[MAX_ACC], acc_empty[MAX_ACC];
+  uint64_t done;                                   // every MMA this CTA has issued is complete
   uint32_t tmem_base;
   int abort;
   __align__(16) float rn_col[EPI_WARPS][128];    // inverse norms of this warp's columns
@@ -239,14 +243,59 @@ __device__ __forceinline__ void gram_chunk(const uint32_t (&v)[32], const float 
   }
 }
 
+// Labels of a group of 32 tokens (lane = token) whose nearest centres are final, formed by the last epilogue
+// warp of the rows x centres pass to finish the group: a survivor takes its nearest centre's cluster (a centre
+// its own), a pruned token that cluster iff the distance is strictly below alpha * d_c (Eq. 8-9), else -1.
+// The group's members per cluster are added to the table of its 256-token block and to the cluster sizes
+// (integer adds: the sums do not depend on the order in which groups finish).
+// r: the token's position among the survivors (< 0: pruned); own_cid: its cluster id if it is a centre, else -1
+// (both known before the pass, so that only the nearest centre has to be fetched here).
+__device__ __forceinline__ void label_group(const ImgDesc &im, int i, int lane, int C, int r, int own_cid) {
+  int lab = -1, joined = 0, dropped = 0, band = 0;
+  if (i < im.N) {
+    const unsigned long long pk = __ldcg(im.best + i);
+    lab = (int)(pk & 0xFFFFFFFFull);
+    const float dd = __uint_as_float((uint32_t)(pk >> 32));
+    if (r >= 0) {
+      if (own_cid >= 0) lab = own_cid;
+    } else {
+      if (DistF::in_band_t(dd, im)) ++band;
+      if (DistF::below_t(dd, im)) ++joined; else { lab = -1; ++dropped; }
+    }
+    if (lab >= C || lab < -1) lab = -1;             // only after a failed earlier stage
+    im.label[i] = lab;
+    if (im.label_user) im.label_user[i] = lab;
+  }
+  const unsigned same = __match_any_sync(0xffffffffu, lab);
+  if (lab >= 0 && lane == __ffs(same) - 1) {
+    const int len = __popc(same), b = i / kListBlock;
+    // 16-bit cell (c, b) of the table, added to through the 32-bit word that holds it (a cell stays <= 256)
+    uint32_t *word = reinterpret_cast<uint32_t *>(im.cnt_cb) + (((size_t)lab * im.nbp + b) >> 1);
+    atomicAdd(word, (uint32_t)len << (16 * (b & 1)));
+    atomicAdd(&im.csize[lab], len);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    joined += __shfl_xor_sync(0xffffffffu, joined, o);
+    dropped += __shfl_xor_sync(0xffffffffu, dropped, o);
+    band += __shfl_xor_sync(0xffffffffu, band, o);
+  }
+  if (lane == 0) {
+    if (joined) atomicAdd(&im.cnt[PACT_CNT_R], joined);
+    if (dropped) atomicAdd(&im.cnt[PACT_CNT_DISCARDED], dropped);
+    if (band) atomicAdd(&im.cnt[PACT_CNT_BAND_ADC], band);
+  }
+}
+
 // The epilogue of one accumulator tile for one warp: the warp's 32 rows (tensor-memory lanes) of the 128-row
 // block tmi against HALF columns from cbase on.  Waits for the accumulator, reads it 32 columns at a time and
 // applies the mode's arithmetic; arrive() is called once the accumulator has been read.  skip: the warp only
 // waits and releases (a block below the diagonal of the all-pairs pass).  Returns false when the wait ran out.
-template <int MODE, int HALF, typename Arrive>
+template <int MODE, int HALF, bool WAIT_MIN = false, typename Arrive>
 __device__ __forceinline__ bool epi_tile(const ImgDesc &im, int kept_rows, int tmi, int cbase, bool skip, int nrows,
                                          int ncols, uint32_t taddr, uint64_t *acc_full, uint32_t parity, float *rn_col,
-                                         uint32_t *tr, int lane, int qd, int &band, float &mx, Arrive arrive) {
+                                         uint32_t *tr, int lane, int qd, int &band, float &mx, Arrive arrive,
+                                         unsigned long long &seen) {
   // inverse norms of this warp's columns and of this lane's row (in flight while the MMAs run)
   const float *rn_src = MODE == MODE_GRAM ? im.rnk : (MODE == MODE_SPREAD ? im.rn : im.rnc);
   float4 r4;
@@ -354,7 +403,8 @@ __device__ __forceinline__ bool epi_tile(const ImgDesc &im, int kept_rows, int t
     if (MODE == MODE_GRAM) atomicAdd(&im.rho_fix[row], rowsum);
     else if (MODE == MODE_ASSIGN && bd <= 2.0f) {
       const unsigned long long pk = ((unsigned long long)__float_as_uint(bd) << 32) | (unsigned)bi;
-      atomicMin(&im.best[kept_rows ? im.kept_idx[row] : row], pk);
+      const unsigned long long old = atomicMin(&im.best[kept_rows ? im.kept_idx[row] : row], pk);
+      if (WAIT_MIN) seen |= old;                   // the caller waits for the value: the minimum is then in place
     }
   }
   return true;
@@ -363,7 +413,8 @@ __device__ __forceinline__ bool epi_tile(const ImgDesc &im, int kept_rows, int t
 }  // namespace
 
 // grid (X, B), 320 threads, dynamic smem = TileCfg<BN>::SMEM.
-// kept_rows (assignment only): rows are the gathered survivors (Kp, rnk) instead of all tokens.
+// kept_rows (assignment only), bit 0: rows are the gathered survivors (Kp, rnk) instead of all tokens;
+// bit 1: the labels, cluster sizes and per-block member counts are formed here as groups of rows finish.
 template <int MODE, int BN>
 __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant__ Batch bt,
                                                            const __grid_constant__ TmapSet tm, int kept_rows) {
@@ -382,6 +433,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
     for (int a = 0; a < NACC; ++a) { mbar_init(&sh.acc_full[a], 1); mbar_init(&sh.acc_empty[a], EPI_WARPS); }
+    mbar_init(&sh.done, 1);
     sh.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -396,7 +448,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
   int nrows, ncols;
   if (MODE == MODE_GRAM) { nrows = *im.q_ptr; ncols = nrows; }
   else if (MODE == MODE_SPREAD) { nrows = im.N; ncols = im.N; }
-  else { nrows = kept_rows ? *im.q_ptr : im.N; ncols = *im.C_ptr; }
+  else { nrows = (kept_rows & 1) ? *im.q_ptr : im.N; ncols = *im.C_ptr; }
   const int ntm = (nrows + BM - 1) / BM, ntn = (ncols + BN - 1) / BN;
   const int ntiles = tile_count<MODE>(ntm, ntn);
   const bool active = (int)blockIdx.x < ntiles;       // CTAs without a tile only give their tensor memory back
@@ -461,6 +513,9 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
         if (ok) umma_commit(&sh.acc_full[a]);      // accumulator complete
         ++tcount;
       }
+      // whatever way the loop ended, no MMA may still be running when the tensor memory is given back
+      umma_commit(&sh.done);
+      if (!mbar_wait(&sh.done, 0)) ok = false;
       if (!ok) atomicExch(&sh.abort, 1);
     }
   } else {
@@ -474,6 +529,35 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
     int band = 0;
     bool ok = true;
     float mx = 0.f;                                 // largest distance seen by this lane (MODE_SPREAD)
+    // Labels (rows x centres pass with bit 1 of kept_rows): a group of 32 tokens is final once `need` warps
+    // (every column tile, every column half) have put their nearest centres in place; each warp draws a
+    // ticket per group and the one that draws the last labels the group.  The tickets of up to kPend tiles
+    // are drawn together, so that a warp waits for its atomics to land once, not once per tile.
+    constexpr int kPend = 4;
+    const int need = (MODE == MODE_ASSIGN && (kept_rows & 2)) ? ntn * (EPI_WARPS / 4) : 0;
+    int pend_tmi[kPend], pend_r[kPend], pend_cid[kPend], npend = 0;
+    unsigned long long seen = 0ull;                 // previous values of the minima this lane has updated
+    auto flush_labels = [&]() {
+      // Every lane's atomic minima have returned, i.e. are in place, once their return values have been used:
+      // the fence then has nothing left to wait for.  (No stored value has distance bits above 2.0f.)
+      const unsigned odd = __ballot_sync(0xffffffffu, seen == 0xFFFFFFFE00000001ull);
+      seen = 0ull;
+      __threadfence();
+      int mine = 0;
+      if (lane < npend && odd == 0u) {
+        int tmi_l = pend_tmi[0];
+#pragma unroll
+        for (int k = 1; k < kPend; ++k) if (lane == k) tmi_l = pend_tmi[k];
+        mine = atomicAdd(&im.rtick[tmi_l * (BM / 32) + qd], 1) == need - 1;
+      }
+      const unsigned lastmask = __ballot_sync(0xffffffffu, mine);
+      if (lastmask) __threadfence();
+#pragma unroll
+      for (int k = 0; k < kPend; ++k)
+        if (k < npend && ((lastmask >> k) & 1u))
+          label_group(im, pend_tmi[k] * BM + qd * 32 + lane, lane, ncols, pend_r[k], pend_cid[k]);
+      npend = 0;
+    };
     for (int tile = blockIdx.x; ok && tile < ntiles; tile += gridDim.x) {
       int tmi, tni;
       tile_at<MODE>(tile, ntm, ntn, tmi, tni);
@@ -481,11 +565,27 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
       const uint32_t a = tcount % NACC;
       const int cbase = tni * BN + half * HALF;     // first column of this warp
       const uint32_t taddr = tmem_base + a * BN + half * HALF + ((uint32_t)(qd * 32) << 16);
-      ok = epi_tile<MODE, HALF>(im, kept_rows, tmi, cbase, false, nrows, ncols, taddr, &sh.acc_full[a], (tcount / NACC) & 1,
-                                rn_col, tr, lane, qd, band, mx, [&]() { mbar_arrive(&sh.acc_empty[a]); });
+      if (MODE == MODE_ASSIGN && need > 0) {
+        // what the labels of this warp's 32 tokens need besides the nearest centre (known before the pass)
+        const int row = tmi * BM + qd * 32 + lane;
+        int r = -1, own = -1;
+        if (row < nrows) {
+          r = im.slot[row];
+          if (r >= 0 && ((im.cmask[r >> 5] >> (r & 31)) & 1u)) own = im.cid[r];
+        }
+        pend_tmi[npend] = tmi; pend_r[npend] = r; pend_cid[npend] = own;
+      }
+      if (need > 0)
+        ok = epi_tile<MODE, HALF, true>(im, kept_rows & 1, tmi, cbase, false, nrows, ncols, taddr, &sh.acc_full[a], (tcount / NACC) & 1,
+                                        rn_col, tr, lane, qd, band, mx, [&]() { mbar_arrive(&sh.acc_empty[a]); }, seen);
+      else
+        ok = epi_tile<MODE, HALF>(im, kept_rows & 1, tmi, cbase, false, nrows, ncols, taddr, &sh.acc_full[a], (tcount / NACC) & 1,
+                                  rn_col, tr, lane, qd, band, mx, [&]() { mbar_arrive(&sh.acc_empty[a]); }, seen);
       if (!ok) break;
       ++tcount;
+      if (MODE == MODE_ASSIGN && need > 0 && ++npend == kPend) flush_labels();
     }
+    if (MODE == MODE_ASSIGN && need > 0 && ok && npend > 0) flush_labels();
     if (!ok) atomicExch(&sh.abort, 1);
     if (MODE == MODE_GRAM && band) atomicAdd(&im.cnt[PACT_CNT_BAND_DC], band);
     if (MODE == MODE_SPREAD) {
@@ -569,6 +669,7 @@ __device__ __forceinline__ void umma_commit_pair(uint64_t *bar) {
 
 struct SharedPair {
   uint64_t full[PSTAGES], empty[PSTAGES], acc_full[PNACC], acc_empty[PNACC];
+  uint64_t done;                                   // every MMA of the pair is complete (signalled in both CTAs)
   uint32_t tmem_base;
   int abort;
   __align__(16) float rn_col[EPI_WARPS][128];
@@ -593,6 +694,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_pair(const __grid_constant
   if (threadIdx.x == 0) {
     for (int s = 0; s < PSTAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
     for (int a = 0; a < PNACC; ++a) { mbar_init(&sh.acc_full[a], 1); mbar_init(&sh.acc_empty[a], 2 * EPI_WARPS); }
+    mbar_init(&sh.done, 1);
     sh.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -608,7 +710,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_pair(const __grid_constant
   int nrows, ncols;
   if (MODE == MODE_GRAM) { nrows = *im.q_ptr; ncols = nrows; }
   else if (MODE == MODE_SPREAD) { nrows = im.N; ncols = im.N; }
-  else { nrows = kept_rows ? *im.q_ptr : im.N; ncols = *im.C_ptr; }
+  else { nrows = (kept_rows & 1) ? *im.q_ptr : im.N; ncols = *im.C_ptr; }
   const int nti = (nrows + 2 * BM - 1) / (2 * BM), ntj = (ncols + PBN - 1) / PBN;
   const int ntiles = tile_count<MODE>(nti, ntj);
   const int P = gridDim.x >> 1, pr = blockIdx.x >> 1;
@@ -673,8 +775,11 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_pair(const __grid_constant
         if (ok) umma_commit_pair(&sh.acc_full[a]); // accumulator complete, in both CTAs
         ++tcount;
       }
+      umma_commit_pair(&sh.done);                  // both CTAs learn that no MMA is running any more
       if (!ok) atomicExch(&sh.abort, 1);
     }
+    // whatever way the loop ended, no MMA may still be running when the tensor memory is given back
+    if (lane == 0 && !mbar_wait(&sh.done, 0)) atomicExch(&sh.abort, 1);
   } else {
     // ---------------- epilogue (each CTA for its 128 rows) ----------------
     const int ew = warp - 2;
@@ -686,6 +791,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_pair(const __grid_constant
     int band = 0;
     bool ok = true;
     float mx = 0.f;
+    unsigned long long unused_seen = 0ull;
     for (int tile = pr; ok && tile < ntiles; tile += P) {
       int I, J;
       tile_at<MODE>(tile, nti, ntj, I, J);
@@ -697,7 +803,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_pair(const __grid_constant
       const uint32_t taddr = tmem_base + a * PBN + half * 128 + ((uint32_t)(qd * 32) << 16);
       const uint32_t rel = map_to_rank(smem_u32(&sh.acc_empty[a]), 0);
       ok = epi_tile<MODE, 128>(im, kept_rows, R, cbase, skip, nrows, ncols, taddr, &sh.acc_full[a], (tcount / PNACC) & 1,
-                               rn_col, tr, lane, qd, band, mx, [&]() { mbar_arrive_remote(rel); });
+                               rn_col, tr, lane, qd, band, mx, [&]() { mbar_arrive_remote(rel); }, unused_seen);
       if (!ok) break;
       ++tcount;
     }
@@ -828,7 +934,7 @@ cudaError_t launch_gram_umma(const Batch &bt, int maxN, const ClusterCfg &cfg, c
   return launch_k(k_tiles_umma<MODE_GRAM, kGramBN>, grid, dim3(THREADS), TileCfg<kGramBN>::SMEM, st, true, bt, tm, 0);
 }
 
-cudaError_t launch_assign_umma(const Batch &bt, int maxN, bool kept_rows, const ClusterCfg &cfg, cudaStream_t st) {
+cudaError_t launch_assign_umma(const Batch &bt, int maxN, bool kept_rows, const ClusterCfg &cfg, cudaStream_t st, bool labels) {
   TmapSet tm;
   for (int b = 0; b < bt.B; ++b) {
     const ImgDesc &im = bt.img[b];
@@ -839,7 +945,7 @@ cudaError_t launch_assign_umma(const Batch &bt, int maxN, bool kept_rows, const 
   }
   const long long tiles = (long long)((maxN + BM - 1) / BM) * ((maxN + kWideBN - 1) / kWideBN);
   dim3 grid(umma_grid_x(tiles, bt.B, cfg.sm_count), bt.B);
-  return launch_k(k_tiles_umma<MODE_ASSIGN, kWideBN>, grid, dim3(THREADS), TileCfg<kWideBN>::SMEM, st, true, bt, tm, kept_rows ? 1 : 0);
+  return launch_k(k_tiles_umma<MODE_ASSIGN, kWideBN>, grid, dim3(THREADS), TileCfg<kWideBN>::SMEM, st, true, bt, tm, (kept_rows ? 1 : 0) | (labels && !kept_rows ? 2 : 0));
 }
 
 // every layer of the batch is one "image": rows and columns are all N keys of K_clu

@@ -264,6 +264,128 @@ __global__ void __launch_bounds__(kListBlock) k_lists(const __grid_constant__ Ba
   }
 }
 
+// ---- member records from finished labels ----------------------------------------------------------
+// grid (ceil(maxN / 256), B), 256 threads.  The rows x centres pass on the tensor cores has already written
+// the labels, the cluster sizes and cnt_cb (members of cluster c in token block b) as its groups of rows
+// finished; what is left is the second part of k_lists: the member of cluster c that is token i of block b
+// belongs at  member_off[c] + (members of c in the blocks before b) + (members of c before i in block b).
+__global__ void __launch_bounds__(kListBlock) k_members(const __grid_constant__ Batch bt) {
+  const ImgDesc &im = bt.img[blockIdx.y];
+  TL_SCOPE(im, 8);
+  // the number of clusters was final before the rows x centres pass began, and this kernel cannot start before
+  // every CTA of that pass has begun: it may be read ahead of the wait
+  const int C = min(ld_cg_i32(im.C_ptr), im.Np);
+  pdl_wait();
+  pdl_trigger();
+  const int N = im.N;
+  const int nblk = (N + kListBlock - 1) / kListBlock;
+  const int b = blockIdx.x, t = threadIdx.x, lane = t & 31, w = t >> 5;
+  if (b >= nblk) return;
+  __shared__ __align__(16) int slab[kListBlock];
+  __shared__ int excl[kScanTile];
+  __shared__ int wsum[kListBlock / 32];
+  __shared__ int s_carry;
+  const int i = b * kListBlock + t;
+  int c = -1;
+  if (i < N) {
+    if (C > 0) c = ld_cg_i32(&im.label[i]);
+    else {                                           // no centre at all (a failed earlier stage): nothing was labelled
+      im.label[i] = -1;
+      if (im.label_user) im.label_user[i] = -1;
+    }
+    if (c >= C || c < -1) c = -1;
+  }
+  const bool valid = c >= 0;
+  slab[t] = c;
+  // in flight while the block is searched: the counts of the earlier blocks, the cluster's size, the sizes to scan
+  uint4 cb[4];
+  int size = 0;
+  const uint4 *row = reinterpret_cast<const uint4 *>(im.cnt_cb + (size_t)(valid ? c : 0) * im.nbp);
+#pragma unroll
+  for (int v = 0; v < 4; ++v) cb[v] = (valid && v * 8 < b) ? __ldcg(row + v) : make_uint4(0u, 0u, 0u, 0u);
+  if (valid) size = ld_cg_i32(&im.csize[c]);
+  int v8[8];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const int cc = t * 8 + k;
+    v8[k] = cc < C ? ld_cg_i32(&im.csize[cc]) : 0;
+  }
+  __syncthreads();
+  TL_POINT(im, 13);
+  int place = 0;                                     // members of c before token i in this block
+  if (valid) {
+    const int4 *s4 = reinterpret_cast<const int4 *>(slab);
+    const int full = t >> 2;
+    for (int u = 0; u < full; ++u) {
+      const int4 x = s4[u];
+      place += (x.x == c) + (x.y == c) + (x.z == c) + (x.w == c);
+    }
+    const int4 x = s4[full];
+    place += ((t & 3) > 0 && x.x == c) + ((t & 3) > 1 && x.y == c) + ((t & 3) > 2 && x.z == c);
+  }
+  int before = 0;
+#pragma unroll
+  for (int v = 0; v < 4; ++v) {
+    const uint32_t xs[4] = {cb[v].x, cb[v].y, cb[v].z, cb[v].w};
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+      if (v * 8 + k < b) before += (int)((xs[k >> 1] >> ((k & 1) * 16)) & 0xFFFFu);
+  }
+  if (valid)
+    for (int v = 4; v * 8 < b; ++v) {                // more than 32 token blocks
+      const uint4 x = __ldcg(row + v);
+      const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+      for (int k = 0; k < 8; ++k)
+        if (v * 8 + k < b) before += (int)((xs[k >> 1] >> ((k & 1) * 16)) & 0xFFFFu);
+    }
+  // member_off[c] = cluster sizes below c, scanned kScanTile at a time
+  if (t == 0) s_carry = 0;
+  __syncthreads();
+  int moff = 0;
+  for (int base = 0; base < C; base += kScanTile) {
+    int s = 0;
+    if (base > 0) {
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int cc = base + t * 8 + k;
+        v8[k] = cc < C ? ld_cg_i32(&im.csize[cc]) : 0;
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < 8; ++k) s += v8[k];
+    int x = s;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, x, o);
+      if (lane >= o) x += y;
+    }
+    if (lane == 31) wsum[w] = x;
+    __syncthreads();
+    int off = s_carry;
+    for (int k = 0; k < w; ++k) off += wsum[k];
+    int run = off + x - s;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { excl[t * 8 + k] = run; run += v8[k]; }
+    __syncthreads();
+    if (valid && c >= base && c < base + kScanTile) moff = excl[c - base];
+    if (t == kListBlock - 1) s_carry = run;
+    __syncthreads();
+  }
+  if (b == 0 && t == 0) im.cnt[20] = s_carry;        // members in all clusters
+  TL_POINT(im, 14);
+  if (!valid) return;
+  int pos = moff + before + place;
+  pos = max(0, min(pos, N - 1));                     // in bounds whatever an aborted stage left behind
+  im.members[pos] = make_int4(i, c, moff, size);
+  if (before == 0 && place == 0) {                   // first member of the cluster: the row's bookkeeping
+    const int dst = im.vis_start + c;
+    if (im.P_out) im.P_out[dst] = im.P[im.vis_start + min(max(im.cidx_ptr[c], 0), N - 1)];
+    if (im.size_out) im.size_out[dst] = size;
+    if (im.logw_out) im.logw_out[dst] = logf((float)size);   // Eq. 11: log of the token weight
+  }
+}
+
 // ---- Eq. 10 ------------------------------------------------------------------------------------------
 // Grid (X, B), kMrgThreads threads, two CTAs per SM.  Work items are the member records in cluster order
 // followed by the text rows; CTA x takes items [x per, (x + 1) per).  A thread owns VPL groups of 8 columns
@@ -279,10 +401,17 @@ constexpr int kMrgTile = 256;                       // records staged in shared 
 constexpr int kMrgCtasPerSm = 2;
 constexpr int kMrgRingBytes = 160 * 1024 / kMrgCtasPerSm;   // rows in flight per CTA
 
+#ifdef PACT_TL_MERGE
+#define TL_MRG(im, kid) TL_POINT_IF(im, kid, threadIdx.x == 0)
+#else
+#define TL_MRG(im, kid)
+#endif
 template <typename T, typename O, int VPL, int DEPTH>
 __global__ void __launch_bounds__(kMrgThreads, kMrgCtasPerSm) k_merge(const __grid_constant__ Batch bt) {
   const ImgDesc &im = bt.img[blockIdx.y];
   TL_SCOPE(im, 9);
+  // final since the centre selection, which is complete before any kernel after it can start
+  const int C = min(ld_cg_i32(im.C_ptr), im.Np);
   pdl_wait();
   pdl_trigger();
   const int t = threadIdx.x;
@@ -290,7 +419,6 @@ __global__ void __launch_bounds__(kMrgThreads, kMrgCtasPerSm) k_merge(const __gr
   __shared__ int s_dst[kMrgTile];                   // output row
   __shared__ float s_inv[kMrgTile];                 // 1 / size (1 for text rows and centre-only merging)
   __shared__ int s_last;
-  const int C = min(*im.C_ptr, im.Np);
   const int n_text = im.n_total - im.N;
   const int d = bt.d, ng = d / 8;
   const bool center_only = (im.flags & PACT_FLAG_CENTER_ONLY) != 0;
@@ -449,6 +577,7 @@ __global__ void __launch_bounds__(kMrgThreads, kMrgCtasPerSm) k_merge(const __gr
       s_inv[t] = inv;
     }
     __syncthreads();
+    TL_MRG(im, 10);
     for (int j = 0; j < DEPTH; ++j) issue(j, tn);
 #pragma unroll 1
     for (int j = 0; j < tn; ++j) {
@@ -456,6 +585,7 @@ __global__ void __launch_bounds__(kMrgThreads, kMrgCtasPerSm) k_merge(const __gr
       issue(j + DEPTH, tn);
     }
   }
+  TL_MRG(im, 11);
   if (cur_c < 0) return;                             // an empty range
   const bool goes_on = cur_off + cur_size > hi;
   if (head_open) {                                   // one cluster covers the whole range
@@ -489,6 +619,11 @@ cudaError_t launch_lists(const Batch &bt, int maxN, bool bf16, bool from_best, i
     return launch_lists_t<float, true>(bt, maxN, spin_limit, st);
   }
   return launch_lists_t<float, false>(bt, maxN, spin_limit, st);
+}
+
+cudaError_t launch_members(const Batch &bt, int maxN, cudaStream_t st) {
+  const dim3 grid((maxN + kListBlock - 1) / kListBlock, bt.B);
+  return launch_k(k_members, grid, dim3(kListBlock), 0, st, true, bt);
 }
 
 int lists_kernels(int maxN, int B) {
