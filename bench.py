@@ -31,6 +31,15 @@ N_COPIES = 4          # input copies rotated between steps so that no step finds
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
 # (workload, kernel) -> bytes; absent = not captured for the kernel as it stands
 NCU_TRAFFIC: dict = {
+    ("single_image", "qsum"): 7.49e6,
+    ("single_image", "tokens"): 59.78e6 + 0.23e6,
+    ("single_image", "scores"): 0.34e6,
+    ("single_image", "select"): 3.86e6,
+    ("single_image", "gram_density"): 3.92e6,
+    ("single_image", "centers"): 2.74e6,
+    ("single_image", "assign"): 8.79e6,
+    ("single_image", "label_lists"): 0.11e6,
+    ("single_image", "merge"): 52.33e6 + 0.39e6,
 }
 
 
@@ -488,7 +497,8 @@ def main():
     t_roof = max(t_hbm, t_tc) * B
     n_qcols = wl.n_qh * wl.d_h
     alg = {   # algorithmic bytes (hbm) or flops (tensor) of one launch of each kernel, image 0 scaled by B
-        "euti": ("hbm", img0.N * d * 2.0 + img0.N * d_k * 2.0 + img0.N * n_qcols * 2.0 + q * d_k * 2.0),
+        "qsum": ("hbm", img0.N * n_qcols * 2.0),
+        "tokens": ("hbm", img0.N * d * 2.0 + img0.N * d_k * 2.0),
         "gram_density": ("tensor", 2.0 * d_k * (q * (q + 1) / 2)),
         "assign": ("tensor", 2.0 * d_k * img0.N * Cn),
         "merge": ("hbm", (q + r) * d * 2.0 + Cn * d * 2.0 + 2 * T * d * 2.0),

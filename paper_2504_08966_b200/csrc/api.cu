@@ -9,7 +9,7 @@
 
 using namespace pact;
 
-constexpr int kProfStages = 6;
+constexpr int kProfStages = 9;
 
 struct pact_ctx {
   int d, n_qh, n_kvh, d_h, d_k, n_qcols;
@@ -33,7 +33,8 @@ struct pact_graph {
   int kernels;             // kernels one replay launches
 };
 
-static const char *const kStageNames[kProfStages] = {"euti", "gram_density", "centers", "assign", "label_lists", "merge"};
+static const char *const kStageNames[kProfStages] = {"qsum", "tokens", "scores", "select", "gram_density", "centers",
+                                                    "assign", "label_lists", "merge"};
 
 namespace {
 
@@ -556,7 +557,10 @@ pact_status pact_reduce(pact_ctx *ctx, const pact_image *imgs, int B, const pact
       return cudaEventRecord(ctx->ev[stage], st);
     };
     if (ctx->prof_on && b0 == 0) CK(cudaEventRecord(ctx->ev[0], st));
-    CK(launch_euti(bt, cmaxN, bf, 0, st));  CK(mark());
+    struct MarkFn {
+      static cudaError_t call(void *p) { return (*static_cast<decltype(mark) *>(p))(); }
+    };
+    CK(launch_euti(bt, cmaxN, bf, 0, st, ctx->prof_on ? &MarkFn::call : nullptr, &mark));  CK(mark());
     if (ctx->umma) CK(launch_gram_umma(bt, cmaxN, ctx->ccfg, st));
     else launch_gram(bt, cmaxN, bf, ctx->ccfg, st);
     CK(mark());

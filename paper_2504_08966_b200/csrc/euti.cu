@@ -911,18 +911,21 @@ static int qsum_row_blocks(int ncg, int B) {
 }
 
 template <typename T>
-static cudaError_t launch_euti_t(const Batch &bt, int maxN, int mode, cudaStream_t st) {
+static cudaError_t launch_euti_t(const Batch &bt, int maxN, int mode, cudaStream_t st, StageMark mark, void *mark_arg) {
   constexpr int V = Vec<T>::N;
   const int ncg = (bt.n_qcols / V + 7) / 8;
   const int RP = qsum_row_blocks(ncg, bt.B);
   cudaError_t e = launch_k(k_qsum<T>, dim3(ncg * RP, bt.B), dim3(kQsumThreads), 0, st, false, bt, RP, mode == 0 ? 1 : 0);
   if (e != cudaSuccess) return e;
+  if (mark && (e = mark(mark_arg)) != cudaSuccess) return e;
   const size_t sm_tok = (size_t)(bt.n_qcols + kRowsPerCta * bt.n_qh) * sizeof(double);
   e = launch_k(k_tokens<T>, dim3((maxN + kRowsPerCta - 1) / kRowsPerCta, bt.B), dim3(kTokThreads), sm_tok, st, true, bt);
   if (e != cudaSuccess) return e;
+  if (mark && (e = mark(mark_arg)) != cudaSuccess) return e;
   e = launch_k(k_scores, dim3((maxN + 255) / 256, bt.B), dim3(256), 0, st, true, bt, mode == 0 ? 1 : 0);
   if (e != cudaSuccess) return e;
   if (mode == 0) {
+    if (mark && (e = mark(mark_arg)) != cudaSuccess) return e;
     size_t keys = (size_t)maxN * sizeof(uint32_t);
     const int in_smem = keys <= 96 * 1024;
     if (!in_smem) keys = 0;
@@ -936,8 +939,9 @@ static cudaError_t launch_euti_t(const Batch &bt, int maxN, int mode, cudaStream
   return cudaGetLastError();
 }
 
-cudaError_t launch_euti(const Batch &bt, int maxN, bool bf16, int mode, cudaStream_t st) {
-  return bf16 ? launch_euti_t<__nv_bfloat16>(bt, maxN, mode, st) : launch_euti_t<float>(bt, maxN, mode, st);
+cudaError_t launch_euti(const Batch &bt, int maxN, bool bf16, int mode, cudaStream_t st, StageMark mark, void *mark_arg) {
+  return bf16 ? launch_euti_t<__nv_bfloat16>(bt, maxN, mode, st, mark, mark_arg)
+              : launch_euti_t<float>(bt, maxN, mode, st, mark, mark_arg);
 }
 
 int euti_kernels(int mode) { return mode == 0 ? 4 : 3; }

@@ -52,7 +52,10 @@ inline cudaError_t launch_coop(void (*kernel)(KArgs...), dim3 grid, dim3 block, 
 
 // Algorithm 1.  mode 0: scores, threshold, lists, survivor keys (four kernels; the first also clears what later
 // kernels accumulate into); mode 1: scores only (three kernels).
-cudaError_t launch_euti(const Batch &bt, int maxN, bool bf16, int mode, cudaStream_t st);
+// mark (optional) is called between the kernels of the group (the per-kernel timing of a profiled call)
+typedef cudaError_t (*StageMark)(void *);
+cudaError_t launch_euti(const Batch &bt, int maxN, bool bf16, int mode, cudaStream_t st, StageMark mark = nullptr,
+                        void *mark_arg = nullptr);
 int euti_kernels(int mode);
 // threshold + ordered compaction; gather: also copy the survivor keys and clear the accumulators
 void launch_select_gather(const Batch &bt, int maxN, bool bf16, bool gather, cudaStream_t st);
