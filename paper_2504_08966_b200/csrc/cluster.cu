@@ -7,10 +7,6 @@
 #include <cooperative_groups.h>
 
 #include "kernels.cuh"
-#if defined(PACT_TL_EUTI) || defined(PACT_TL_MERGE)
-#undef TL_POINT
-#define TL_POINT(im, kid)
-#endif
 
 namespace pact {
 

@@ -430,12 +430,6 @@ constexpr int kSelBits = 10;                  // key bits per pass of the select
 constexpr int kSelPerThread = (1 << kSelBits) / kSelThreads;
 static_assert(kHistPerThread % 4 == 0 && kHistPerThread * kSelThreads == (1 << kHistBits), "histogram split");
 
-#ifdef PACT_TL_EUTI
-#define TL_DBG(im, kid) TL_POINT(im, kid)
-#else
-#define TL_DBG(im, kid)
-#endif
-
 struct SelShared {
   int hist[1 << kSelBits];
   int wtot[kSelWarps], wtot2[kSelWarps];
@@ -464,7 +458,6 @@ __device__ __forceinline__ uint32_t euti_threshold(const ImgDesc &im, const uint
       const int y = __shfl_up_sync(0xffffffffu, incl, o);
       if (lane >= o) incl += y;
     }
-    TL_DBG(im, 10);
     if (lane == 31) sh.wtot[w] = incl;
     if (t == 0) { sh.s_bin = -1; sh.s_k = 0; }
 #pragma unroll
@@ -484,7 +477,6 @@ __device__ __forceinline__ uint32_t euti_threshold(const ImgDesc &im, const uint
     }
     __syncthreads();
   }
-  TL_DBG(im, 11);
   if (sh.s_bin < 0) return 0xffffffffu;                 // inconsistent histogram: keep nothing
   if (t == 0) sh.s_prefix = (uint32_t)sh.s_bin << kHistShift;
   __syncthreads();
@@ -535,7 +527,6 @@ __device__ __forceinline__ uint32_t euti_threshold(const ImgDesc &im, const uint
       }
     }
     __syncthreads();
-    TL_DBG(im, hi == kHistShift ? 12 : 13);
     if (lo > 0 && sh.s_cnt == 1) {                      // one key left under the prefix: it is the threshold
       const uint32_t fixed = ~((1u << lo) - 1u), pre2 = sh.s_prefix;
       if (KPT > 0) {
@@ -589,7 +580,6 @@ __device__ __forceinline__ void euti_compact(const Batch &bt, const ImgDesc &im,
   int before0 = 0, q = 0;
 #pragma unroll
   for (int k = 0; k < kSelWarps; ++k) { before0 += sh.wtot[k]; q += sh.wtot2[k]; }
-  TL_DBG(im, 14);
   if (g == 0 && t == 0) {
     im.cnt[PACT_CNT_Q] = q;
     im.cnt[PACT_CNT_M] = N - q;

@@ -14,10 +14,6 @@
 #include <cooperative_groups.h>
 
 #include "kernels.cuh"
-#ifdef PACT_TL_EUTI
-#undef TL_POINT
-#define TL_POINT(im, kid)
-#endif
 
 namespace pact {
 
@@ -401,11 +397,6 @@ constexpr int kMrgTile = 256;                       // records staged in shared 
 constexpr int kMrgCtasPerSm = 2;
 constexpr int kMrgRingBytes = 160 * 1024 / kMrgCtasPerSm;   // rows in flight per CTA
 
-#ifdef PACT_TL_MERGE
-#define TL_MRG(im, kid) TL_POINT_IF(im, kid, threadIdx.x == 0)
-#else
-#define TL_MRG(im, kid)
-#endif
 template <typename T, typename O, int VPL, int DEPTH>
 __global__ void __launch_bounds__(kMrgThreads, kMrgCtasPerSm) k_merge(const __grid_constant__ Batch bt) {
   const ImgDesc &im = bt.img[blockIdx.y];
@@ -577,7 +568,7 @@ __global__ void __launch_bounds__(kMrgThreads, kMrgCtasPerSm) k_merge(const __gr
       s_inv[t] = inv;
     }
     __syncthreads();
-    TL_MRG(im, 10);
+    TL_POINT(im, 15);
     for (int j = 0; j < DEPTH; ++j) issue(j, tn);
 #pragma unroll 1
     for (int j = 0; j < tn; ++j) {
@@ -585,7 +576,6 @@ __global__ void __launch_bounds__(kMrgThreads, kMrgCtasPerSm) k_merge(const __gr
       issue(j + DEPTH, tn);
     }
   }
-  TL_MRG(im, 11);
   if (cur_c < 0) return;                             // an empty range
   const bool goes_on = cur_off + cur_size > hi;
   if (head_open) {                                   // one cluster covers the whole range
