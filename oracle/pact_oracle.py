@@ -336,7 +336,10 @@ def pact_reduce(H, K_euti, Q_euti, K_clu, P, vis_start, N, n_qh, n_kvh, lam, d_c
                                np.ones(n_total - vis_start - N, np.int64)])
     t = reinc_threshold(alpha, dc)
     Dp = cosine_distance(K_clu[pruned], K_clu[center_token]) if pruned.size else np.zeros((0, C))
-    frag = fragile_decisions(scores, tau, cl["D"], cl["rho"], cl["order"], dc, cl["D"][:, centers_local], Dp, t)
+    # the threshold in float64: the smallest float64 score that was kept (tau itself is a float32 value, which
+    # differs from the float64 score of the token that defines it by its own rounding)
+    tau64 = float(scores[keep].min()) if keep.any() else float(tau)
+    frag = fragile_decisions(scores, tau64, cl["D"], cl["rho"], cl["order"], dc, cl["D"][:, centers_local], Dp, t)
     return {
         "scores": scores, "scores32": scores32, "tau": tau, "keep": keep, "kept_idx": kept,
         "pruned_idx": pruned, "D": cl["D"], "rho": cl["rho"], "order": cl["order"],
