@@ -32,18 +32,20 @@ __device__ __forceinline__ uint32_t score_key(float s) {
 }
 
 // ---- Eq. 1: column sums of Q -----------------------------------------------------------------------------
-// grid (ncg RP, B), 256 threads (few registers: the CTAs of k_tokens start beside them).  Work item (column
-// group of eight 16-byte vectors, block of rows): thread t takes vector t & 7 of the group and the rows
-// r0 + (t >> 3), + 32, ...; the four row lanes of a warp are added with shuffles, the eight warps through
+// grid (ncg RP, B), 512 threads at no more than 64 registers, on fewer than half of the SMs: a CTA leaves room
+// for one CTA of k_tokens beside it, and the other SMs take two, so that all of them start at once.  Work item
+// (column group of eight 16-byte vectors, block of rows): thread t takes vector t & 7 of the group and the rows
+// r0 + (t >> 3), + 64, ...; the four row lanes of a warp are added with shuffles, the warps through
 // shared memory.  The CTA that finishes a column group's last
 // row block adds the RP partial sums in block order and writes the group's part of the global query, so the
 // result does not depend on which CTA that is.  do_init: the grid also clears what later kernels accumulate
 // into.
-constexpr int kQsumThreads = 256;
+constexpr int kQsumThreads = 512;
+constexpr int kQsumRowLanes = kQsumThreads / 8;
 constexpr int kQsumWarps = kQsumThreads / 32;
 
 template <typename T>
-__global__ void __launch_bounds__(kQsumThreads, 4) k_qsum(const __grid_constant__ Batch bt, int RP, int do_init) {
+__global__ void __launch_bounds__(kQsumThreads, 2) k_qsum(const __grid_constant__ Batch bt, int RP, int do_init) {
   constexpr int V = Vec<T>::N;
   const ImgDesc &im = bt.img[blockIdx.y];
   TL_SCOPE(im, 0);
@@ -76,14 +78,15 @@ __global__ void __launch_bounds__(kQsumThreads, 4) k_qsum(const __grid_constant_
   if (v < nvq) {
     constexpr int UQ = 8;
     const size_t coff = (size_t)v * V;
-    for (int r = r0 + (t >> 3); r < r1; r += 32 * UQ) {
+    for (int r = r0 + (t >> 3); r < r1; r += kQsumRowLanes * UQ) {
       uint4 buf[UQ];
 #pragma unroll
       for (int u = 0; u < UQ; ++u)
-        if (r + u * 32 < r1) buf[u] = ldg_hint(reinterpret_cast<const uint4 *>(Q + (size_t)(r + u * 32) * im.ldQ + coff), pol);
+        if (r + u * kQsumRowLanes < r1)
+          buf[u] = ldg_hint(reinterpret_cast<const uint4 *>(Q + (size_t)(r + u * kQsumRowLanes) * im.ldQ + coff), pol);
 #pragma unroll
       for (int u = 0; u < UQ; ++u) {
-        if (r + u * 32 < r1) {
+        if (r + u * kQsumRowLanes < r1) {
           float x[V];
           widen_vec<T>(buf[u], x);
 #pragma unroll
@@ -172,11 +175,10 @@ __global__ void __launch_bounds__(kTokThreads, 2) k_tokens(const __grid_constant
 
   // the global query is kept transposed, qT[k][vq] = Qglobal[vq * V + k], so that the lanes of a warp,
   // which hold consecutive 16-byte vectors of the key row, read consecutive doubles
-  // first the rows: |h_i| and 1 / |k_i| of the warp's tokens, one token after the other
-#pragma unroll 1
-  for (int i = 0; i < kTokPerWarp; ++i) {
+  // the rows: |h_i| and 1 / |k_i| of one of the warp's tokens
+  auto row_pass = [&](int i) {
     const int tok = r0 + w * kTokPerWarp + i;
-    if (tok >= r1) break;                               // the same for the whole warp
+    if (tok >= r1) return;                              // the same for the whole warp
     uint4 kb[UK];
     const T *kcrow = im.Kc ? reinterpret_cast<const T *>(im.Kc) + (size_t)tok * im.ldKc : nullptr;
     if (kcrow) {
@@ -198,6 +200,20 @@ __global__ void __launch_bounds__(kTokThreads, 2) k_tokens(const __grid_constant
       if (nv > 32 * UK) a += row_sumsq_lane<T, 8>(kcrow, bt.d_k, lane, 32 * UK);
       const double ss = warp_sum(a);
       if (lane == 0) rn_tok<D>(im)[tok] = (rn_t)(1.0 / sqrt(fmax(ss, 1e-40)));
+    }
+  };
+  // first all but the last of the warp's tokens, one after the other
+#pragma unroll 1
+  for (int i = 0; i + 1 < kTokPerWarp; ++i) row_pass(i);
+  // the last token's hidden-state row is asked for now (into the L2) and read after the logits, which are
+  // formed while it is on its way
+  {
+    const int tok = r0 + w * kTokPerWarp + kTokPerWarp - 1;
+    if (tok < r1 && !(im.flags & PACT_FLAG_NO_NORM)) {
+      const char *hrow = reinterpret_cast<const char *>(reinterpret_cast<const T *>(im.H) + (size_t)(im.vis_start + tok) * im.ldH);
+      const int bytes = bt.d * (int)sizeof(T);
+      for (int o = lane * 128; o < bytes; o += 32 * 128)
+        asm volatile("prefetch.global.L2::evict_last [%0];" ::"l"(hrow + o));
     }
   }
   // the global query is kept transposed, qT[k][vq] = Qglobal[vq * V + k], so that the lanes of a warp,
@@ -296,6 +312,7 @@ __global__ void __launch_bounds__(kTokThreads, 2) k_tokens(const __grid_constant
       }
     }
   }
+  row_pass(kTokPerWarp - 1);
   __syncthreads();
   // per head: CTA max, exp, CTA sum; lane = token within the CTA
   for (int j = w; j < n_qh; j += kTokWarps) {
@@ -896,7 +913,8 @@ constexpr size_t kSelectReserve = 4096;      // static shared memory of k_select
 }  // namespace
 
 static int qsum_row_blocks(int ncg, int B) {
-  int RP = 2 * g_sm_count / (ncg * B);         // about two CTAs per SM
+  // CTAs on 7/16 of the SMs (64 of 148): see k_qsum
+  int RP = g_sm_count * 7 / 16 / (ncg * B);
   return RP < 1 ? 1 : (RP > kQPartRows ? kQPartRows : RP);
 }
 
