@@ -246,7 +246,7 @@ __device__ __forceinline__ void gram_chunk(const uint32_t (&v)[32], const float 
 // Labels of a group of 32 tokens (lane = token) whose nearest centres are final, formed by the last epilogue
 // warp of the rows x centres pass to finish the group: a survivor takes its nearest centre's cluster (a centre
 // its own), a pruned token that cluster iff the distance is strictly below alpha * d_c (Eq. 8-9), else -1.
-// The group's members per cluster are added to the table of its 256-token block and to the cluster sizes
+// The group's members per cluster are added to the table of its 128-token block and to the cluster sizes
 // (integer adds: the sums do not depend on the order in which groups finish).
 // r: the token's position among the survivors (< 0: pruned); own_cid: its cluster id if it is a centre, else -1
 // (both known before the pass, so that only the nearest centre has to be fetched here).
@@ -269,7 +269,7 @@ __device__ __forceinline__ void label_group(const ImgDesc &im, int i, int lane, 
   const unsigned same = __match_any_sync(0xffffffffu, lab);
   if (lab >= 0 && lane == __ffs(same) - 1) {
     const int len = __popc(same), b = i / kListBlock;
-    // 16-bit cell (c, b) of the table, added to through the 32-bit word that holds it (a cell stays <= 256)
+    // 16-bit cell (c, b) of the table, added to through the 32-bit word that holds it (a cell stays <= 128)
     uint32_t *word = reinterpret_cast<uint32_t *>(im.cnt_cb) + (((size_t)lab * im.nbp + b) >> 1);
     atomicAdd(word, (uint32_t)len << (16 * (b & 1)));
     atomicAdd(&im.csize[lab], len);

@@ -3,7 +3,7 @@
 // text rows copied around the merged span.
 //
 //   k_lists  labels (reincorporation test of Eq. 8), then a stable counting sort of the tokens by
-//            cluster id: every block of 256 tokens sorts its own, an image-wide barrier, and every
+//            cluster id: every block of 128 tokens sorts its own, an image-wide barrier, and every
 //            token writes one 16-byte record {token, cluster, first member position, cluster size}
 //            at its place in the cluster-sorted member array.  Also P', sizes and log sizes.
 //   k_merge  the member array (followed by the text rows) is cut into one contiguous range per CTA;
@@ -73,8 +73,8 @@ __device__ __forceinline__ float4 ld_cg_f4(const float *p) {
 }
 
 // ---- member lists --------------------------------------------------------------------------------
-// grid (ceil(maxN / 256), B), 256 threads.
-// Part 1: block b sorts its 256 tokens by (cluster id, token), discarded tokens last; the first token of
+// grid (ceil(maxN / 128), B), 128 threads.
+// Part 1: block b sorts its 128 tokens by (cluster id, token), discarded tokens last; the first token of
 //   every run writes the run length to cnt_cb[c][b] (a table that is zero before the kernel) and adds it
 //   to csize[c].
 // Part 2 (after every block of the image has finished part 1): the member in sorted position t of block b
@@ -261,7 +261,7 @@ __global__ void __launch_bounds__(kListBlock) k_lists(const __grid_constant__ Ba
 }
 
 // ---- member records from finished labels ----------------------------------------------------------
-// grid (ceil(maxN / 256), B), 256 threads.  The rows x centres pass on the tensor cores has already written
+// grid (ceil(maxN / 128), B), 128 threads.  The rows x centres pass on the tensor cores has already written
 // the labels, the cluster sizes and cnt_cb (members of cluster c in token block b) as its groups of rows
 // finished; what is left is the second part of k_lists: the member of cluster c that is token i of block b
 // belongs at  member_off[c] + (members of c in the blocks before b) + (members of c before i in block b).
@@ -294,11 +294,12 @@ __global__ void __launch_bounds__(kListBlock) k_members(const __grid_constant__ 
   const bool valid = c >= 0;
   slab[t] = c;
   // in flight while the block is searched: the counts of the earlier blocks, the cluster's size, the sizes to scan
-  uint4 cb[4];
+  constexpr int kCbRegs = 8;                         // rows of cnt_cb of up to 64 token blocks are read at once
+  uint4 cb[kCbRegs];
   int size = 0;
   const uint4 *row = reinterpret_cast<const uint4 *>(im.cnt_cb + (size_t)(valid ? c : 0) * im.nbp);
 #pragma unroll
-  for (int v = 0; v < 4; ++v) cb[v] = (valid && v * 8 < b) ? __ldcg(row + v) : make_uint4(0u, 0u, 0u, 0u);
+  for (int v = 0; v < kCbRegs; ++v) cb[v] = (valid && v * 8 < b) ? __ldcg(row + v) : make_uint4(0u, 0u, 0u, 0u);
   if (valid) size = ld_cg_i32(&im.csize[c]);
   int v8[8];
 #pragma unroll
@@ -321,14 +322,14 @@ __global__ void __launch_bounds__(kListBlock) k_members(const __grid_constant__ 
   }
   int before = 0;
 #pragma unroll
-  for (int v = 0; v < 4; ++v) {
+  for (int v = 0; v < kCbRegs; ++v) {
     const uint32_t xs[4] = {cb[v].x, cb[v].y, cb[v].z, cb[v].w};
 #pragma unroll
     for (int k = 0; k < 8; ++k)
       if (v * 8 + k < b) before += (int)((xs[k >> 1] >> ((k & 1) * 16)) & 0xFFFFu);
   }
   if (valid)
-    for (int v = 4; v * 8 < b; ++v) {                // more than 32 token blocks
+    for (int v = kCbRegs; v * 8 < b; ++v) {          // more token blocks than that
       const uint4 x = __ldcg(row + v);
       const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
