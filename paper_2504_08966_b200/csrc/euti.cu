@@ -912,9 +912,12 @@ size_t g_smem_optin = 48 * 1024;
 constexpr size_t kSelectReserve = 4096;      // static shared memory of k_select_gather, rounded up
 }  // namespace
 
-static int qsum_row_blocks(int ncg, int B) {
-  // CTAs on 7/16 of the SMs (64 of 148): see k_qsum
+static int qsum_row_blocks(int ncg, int B, int maxN) {
+  // CTAs on 7/16 of the SMs (64 of 148) when that leaves a CTA no more than two rounds of loads (1024 rows),
+  // else as many row blocks as that takes: see k_qsum
   int RP = g_sm_count * 7 / 16 / (ncg * B);
+  const int need = (maxN + 1023) / 1024;
+  if (RP < need) RP = need;
   return RP < 1 ? 1 : (RP > kQPartRows ? kQPartRows : RP);
 }
 
@@ -922,7 +925,7 @@ template <typename T>
 static cudaError_t launch_euti_t(const Batch &bt, int maxN, int mode, cudaStream_t st, StageMark mark, void *mark_arg) {
   constexpr int V = Vec<T>::N;
   const int ncg = (bt.n_qcols / V + 7) / 8;
-  const int RP = qsum_row_blocks(ncg, bt.B);
+  const int RP = qsum_row_blocks(ncg, bt.B, maxN);
   cudaError_t e = launch_k(k_qsum<T>, dim3(ncg * RP, bt.B), dim3(kQsumThreads), 0, st, false, bt, RP, mode == 0 ? 1 : 0);
   if (e != cudaSuccess) return e;
   if (mark && (e = mark(mark_arg)) != cudaSuccess) return e;
