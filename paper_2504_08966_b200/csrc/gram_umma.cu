@@ -366,20 +366,36 @@ __device__ __forceinline__ bool epi_tile(const ImgDesc &im, int kept_rows, int t
       }
       if (row_ok) im.adj[(size_t)row * im.Wp + (c0 >> 5)] = bits;
     } else if (MODE == MODE_SPREAD) {
-      // rows and columns past the end hold zero dot products, i.e. distance 1: leave them out
-      const int lim = row_ok ? min(32, ncols - c0) : 0;
-      const int self = row - c0;                 // the pair (i, i) is not a pair
+      // The largest distance of the chunk belongs to its smallest cosine: d = clamp(1 - c) does not increase
+      // with c, in floating point either, so the cosines (dot * rn_i) * rn_j are compared and one distance is
+      // formed per chunk from the smallest.  Rows and columns past the end hold zero dot products,
+      // i.e. distance 1, and the pair (i, i) is not a pair: chunks that hold either take the checked loop.
+      float cmin = 4.0f;
+      const bool plain = c0 + 32 <= ncols && r0 + 32 <= nrows && (c0 + 32 <= r0 || c0 >= r0 + 32);   // uniform
+      if (plain) {
 #pragma unroll
-      for (int k4 = 0; k4 < 32; k4 += 4) {
-        const float4 rn4 = *reinterpret_cast<const float4 *>(rn_col + ch * 32 + k4);
-        const float rnj[4] = {rn4.x, rn4.y, rn4.z, rn4.w};
+        for (int k4 = 0; k4 < 32; k4 += 4) {
+          const float4 rn4 = *reinterpret_cast<const float4 *>(rn_col + ch * 32 + k4);
+          const float rnj[4] = {rn4.x, rn4.y, rn4.z, rn4.w};
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
-          const int k = k4 + kk;
-          const float dd = DistF::dist(__uint_as_float(v[k]), rni, rnj[kk]);
-          if (k < lim && k != self) mx = fmaxf(mx, dd);
+          for (int kk = 0; kk < 4; ++kk) cmin = fminf(cmin, (__uint_as_float(v[k4 + kk]) * rni) * rnj[kk]);
+        }
+      } else {
+        const int lim = row_ok ? min(32, ncols - c0) : 0;
+        const int self = row - c0;
+#pragma unroll
+        for (int k4 = 0; k4 < 32; k4 += 4) {
+          const float4 rn4 = *reinterpret_cast<const float4 *>(rn_col + ch * 32 + k4);
+          const float rnj[4] = {rn4.x, rn4.y, rn4.z, rn4.w};
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk) {
+            const int k = k4 + kk;
+            const float c = (__uint_as_float(v[k]) * rni) * rnj[kk];
+            if (k < lim && k != self) cmin = fminf(cmin, c);
+          }
         }
       }
+      if (cmin < 4.0f) mx = fmaxf(mx, fminf(fmaxf(1.0f - cmin, 0.0f), 2.0f));
     } else {
       const int lim = min(32, ncols - c0);
 #pragma unroll
@@ -634,7 +650,9 @@ __device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank) {
   return r;
 }
 __device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+  // relaxed: the warp has nothing to publish through memory, its reads of the accumulator are complete
+  // (tcgen05.wait::ld) before the arrive is issued, and a release at cluster scope would cost a memory fence
+  asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ void cluster_barrier() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
