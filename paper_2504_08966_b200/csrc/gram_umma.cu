@@ -326,7 +326,7 @@ __device__ __forceinline__ bool epi_tile(const ImgDesc &im, int kept_rows, int t
   if (!mbar_wait_warp(acc_full, parity)) return false;
   tc_fence_after();
   unsigned long long rowsum = 0ull;
-  float bd = 3.0f;                              // best distance so far (assignment); distances are <= 2
+  float bd = 3.0f, bc = -4.0f;                  // distance to the nearest centre of the tile (<= 2) and its cosine
   int bi = 0;
   const float d_c = im.d_c, neg_k = -im.inv_dn_log2e;
   const int r0 = tmi * BM + qd * 32;
@@ -397,6 +397,8 @@ __device__ __forceinline__ bool epi_tile(const ImgDesc &im, int kept_rows, int t
       }
       if (cmin < 4.0f) mx = fmaxf(mx, fminf(fmaxf(1.0f - cmin, 0.0f), 2.0f));
     } else {
+      // the nearest centre of the chunk is the one with the largest cosine (dot * rn_i) * rn_j; the first of
+      // equal cosines wins, i.e. the centre with the lowest index; the distance is formed once per tile
       const int lim = min(32, ncols - c0);
 #pragma unroll
       for (int k4 = 0; k4 < 32; k4 += 4) {
@@ -405,12 +407,13 @@ __device__ __forceinline__ bool epi_tile(const ImgDesc &im, int kept_rows, int t
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk) {
           const int k = k4 + kk;
-          const float dd = DistF::dist(__uint_as_float(v[k]), rni, rnj[kk]);
-          if (k < lim && dd < bd) { bd = dd; bi = c0 + k; }
+          const float c = (__uint_as_float(v[k]) * rni) * rnj[kk];
+          if (k < lim && c > bc) { bc = c; bi = c0 + k; }
         }
       }
     }
   }
+  if (MODE == MODE_ASSIGN && bc > -3.0f) bd = fminf(fmaxf(1.0f - bc, 0.0f), 2.0f);
   // the accumulator may be overwritten once all epilogue warps have read it
   tc_fence_before();
   __syncwarp();
