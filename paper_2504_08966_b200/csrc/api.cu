@@ -561,7 +561,7 @@ pact_status pact_reduce(pact_ctx *ctx, const pact_image *imgs, int B, const pact
       static cudaError_t call(void *p) { return (*static_cast<decltype(mark) *>(p))(); }
     };
     CK(launch_euti(bt, cmaxN, bf, 0, st, ctx->prof_on ? &MarkFn::call : nullptr, &mark));  CK(mark());
-    if (ctx->umma) CK(launch_gram_umma(bt, cmaxN, ctx->ccfg, st));
+    if (ctx->umma) CK(launch_gram_umma(bt, cmaxN, ctx->ccfg, st, cmaxQ));
     else launch_gram(bt, cmaxN, bf, ctx->ccfg, st);
     CK(mark());
     CK(launch_centers(bt, cmaxQ, bf, ctx->ccfg, ctx->sweep_limit, st));  CK(mark());

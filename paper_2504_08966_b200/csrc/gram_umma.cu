@@ -621,13 +621,13 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
   if (threadIdx.x == 0 && sh.abort) atomicMin(&im.cnt[PACT_CNT_STATUS], (int)PACT_ERR_TIMEOUT);
 }
 
-// ---- the largest-distance pass on pairs of CTAs (cta_group::2) ----------------------------------------------
+// ---- tiles on pairs of CTAs (cta_group::2) ----------------------------------------------------------------------
 // Two CTAs of a cluster share one 256 x 256 tile: each holds 128 of its rows (operand A) and 128 of its
 // columns (half of operand B), CTA 0 issues tcgen05.mma.cta_group::2 for both, and each CTA finds its
 // 128 x 256 part of the product in its own tensor memory.  A CTA therefore fetches half as many operand
-// bytes from the L2 per output element as it does alone, and that traffic is what bounds a pass with a light
-// epilogue.  (The all-pairs pass and the rows x centres pass measured slower this way: the first is bound by
-// its epilogue, and both lose more to the coarser tiles than they gain.)
+// bytes from the L2 per output element as it does alone.  The largest-distance pass always runs this way, the
+// all-pairs pass when an SM has six or more 128 x 128 blocks to do (with fewer, the coarser tiles cost a round);
+// the rows x centres pass measured slower this way.
 //   full[s]      in CTA 0: both CTAs' copies of stage s report their bytes there
 //   empty[s]     in each CTA: tcgen05.commit (multicast to both CTAs) once the MMAs have read stage s
 //   acc_full[a]  in each CTA: tcgen05.commit (multicast) once accumulator a is complete
@@ -635,11 +635,18 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
 // Every wait is bounded as in the single-CTA kernel; the CTAs leave together through a cluster barrier, after
 // which nothing is in flight towards either's shared memory.
 constexpr int PBN = 256;                              // tile width of the pair kernel
-constexpr int PSTAGES = 5;
 constexpr int PSTAGE_BYTES = 2 * A_BYTES;             // 128 rows of A and 128 rows of B per CTA and stage
 constexpr int PNACC = TMEM_COLS / PBN;
-constexpr size_t PRING = 1024 + (size_t)PSTAGES * PSTAGE_BYTES;
-template <int MODE> constexpr size_t pair_smem() { return PRING + (MODE == MODE_GRAM ? (size_t)EPI_WARPS * 32 * 36 * 4 : 0); }
+constexpr int PMAX_STAGES = 5;
+// EW epilogue warps per CTA (8 or 16).  The all-pairs pass runs with 16: its epilogue is heavy, and its exchange
+// buffers (one per epilogue warp) leave room for four stages; the others run with 8 and five stages.
+template <int MODE, int EW> struct PairCfg {
+  static constexpr int STAGES = (MODE == MODE_GRAM && EW > 8) ? 4 : 5;
+  static constexpr size_t RING = 1024 + (size_t)STAGES * PSTAGE_BYTES;
+  static constexpr size_t SMEM = RING + (MODE == MODE_GRAM ? (size_t)EW * 32 * 36 * 4 : 0);
+  static constexpr int THREADS = 64 + EW * 32;
+  static constexpr int COLS = PBN / (EW / 4);      // columns of the tile per epilogue warp
+};
 
 __device__ __forceinline__ uint32_t cluster_rank() {
   uint32_t r;
@@ -688,25 +695,28 @@ __device__ __forceinline__ void umma_commit_pair(uint64_t *bar) {
                ::"r"(smem_u32(bar)), "h"((unsigned short)3) : "memory");
 }
 
-struct SharedPair {
-  uint64_t full[PSTAGES], empty[PSTAGES], acc_full[PNACC], acc_empty[PNACC];
+template <int EW> struct SharedPair {
+  uint64_t full[PMAX_STAGES], empty[PMAX_STAGES], acc_full[PNACC], acc_empty[PNACC];
   uint64_t done;                                   // every MMA of the pair is complete (signalled in both CTAs)
   uint32_t tmem_base;
   int abort;
-  __align__(16) float rn_col[EPI_WARPS][128];
+  __align__(16) float rn_col[EW][128];
 };
 
-// grid (2 P, B) in clusters of two CTAs along x, 320 threads, dynamic smem = pair_smem<MODE>().
+// grid (2 P, B) in clusters of two CTAs along x, 64 + 32 EW threads, dynamic smem = PairCfg<MODE, EW>::SMEM.
 // Pair p takes the 256 x 256 tiles p, p + P, ... of the pass; CTA r of the pair owns the 128-row block 2 I + r of
 // tile (I, J).  In the all-pairs pass a tile is wanted when J >= I, and of the tile (I, I) the block (2 I + 1, 2 I)
 // lies below the diagonal and is computed but not used.
-template <int MODE>
-__global__ void __launch_bounds__(THREADS, 1) k_tiles_pair(const __grid_constant__ Batch bt,
-                                                           const __grid_constant__ TmapSet tm, int kept_rows) {
+template <int MODE, int EW>
+__global__ void __launch_bounds__(PairCfg<MODE, EW>::THREADS, 1) k_tiles_pair(const __grid_constant__ Batch bt,
+                                                                              const __grid_constant__ TmapSet tm, int kept_rows) {
+  using PC = PairCfg<MODE, EW>;
+  constexpr int PSTAGES = PC::STAGES;
+  constexpr size_t PRING = PC::RING;
   const ImgDesc &im = bt.img[blockIdx.y];
   TL_SCOPE(im, MODE == MODE_GRAM ? 4 : 6);
   extern __shared__ uint8_t smem_raw[];
-  __shared__ SharedPair sh;
+  __shared__ SharedPair<EW> sh;
   uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_rank();
@@ -714,7 +724,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_pair(const __grid_constant
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < PSTAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
-    for (int a = 0; a < PNACC; ++a) { mbar_init(&sh.acc_full[a], 1); mbar_init(&sh.acc_empty[a], 2 * EPI_WARPS); }
+    for (int a = 0; a < PNACC; ++a) { mbar_init(&sh.acc_full[a], 1); mbar_init(&sh.acc_empty[a], 2 * EW); }
     mbar_init(&sh.done, 1);
     sh.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -805,7 +815,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_pair(const __grid_constant
     // ---------------- epilogue (each CTA for its 128 rows) ----------------
     const int ew = warp - 2;
     const int qd = warp & 3;                        // tensor-memory lane quadrant this warp may read
-    const int half = ew >> 2;                       // which 128 columns of the tile
+    const int half = ew >> 2;                       // which part of the tile's columns
     float *rn_col = sh.rn_col[ew];
     uint32_t *tr = reinterpret_cast<uint32_t *>(ring + PRING - 1024) + ew * (32 * 36);   // all-pairs pass only
     uint32_t tcount = 0;
@@ -819,11 +829,11 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_pair(const __grid_constant
       if (!wanted(I, J)) continue;
       const uint32_t a = tcount % PNACC;
       const int R = 2 * I + (int)rank;              // this CTA's 128-row block
-      const int cbase = J * PBN + half * 128;       // this warp's columns: one 128-column block
+      const int cbase = J * PBN + half * PC::COLS;  // this warp's columns
       const bool skip = MODE == MODE_GRAM && cbase / BM < R;   // below the diagonal
-      const uint32_t taddr = tmem_base + a * PBN + half * 128 + ((uint32_t)(qd * 32) << 16);
+      const uint32_t taddr = tmem_base + a * PBN + half * PC::COLS + ((uint32_t)(qd * 32) << 16);
       const uint32_t rel = map_to_rank(smem_u32(&sh.acc_empty[a]), 0);
-      ok = epi_tile<MODE, 128>(im, kept_rows, R, cbase, skip, nrows, ncols, taddr, &sh.acc_full[a], (tcount / PNACC) & 1,
+      ok = epi_tile<MODE, PC::COLS>(im, kept_rows, R, cbase, skip, nrows, ncols, taddr, &sh.acc_full[a], (tcount / PNACC) & 1,
                                rn_col, tr, lane, qd, band, mx, [&]() { mbar_arrive_remote(rel); }, unused_seen);
       if (!ok) break;
       ++tcount;
@@ -871,17 +881,19 @@ bool umma_supported(int d_k) { return g_encode != nullptr && d_k % BK == 0; }
 
 namespace {
 bool g_pair_ok = false;                               // clusters of two CTAs of the pair kernel can be launched
+bool g_pair_gram_ok = false;                          // ... of its all-pairs form with 16 epilogue warps
 
-template <int MODE>
+template <int MODE, int EW>
 cudaError_t launch_pair(const Batch &bt, const TmapSet &tm, long long tiles, int kept_rows, const ClusterCfg &cfg, bool pdl,
                         cudaStream_t st) {
+  using PC = PairCfg<MODE, EW>;
   long long P = cfg.sm_count / 2 / bt.B;              // one pair per two SMs: all pairs of the batch run at once
   if (P > tiles) P = tiles;
   if (P < 1) P = 1;
   cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3((unsigned)(2 * P), bt.B);
-  lc.blockDim = dim3(THREADS);
-  lc.dynamicSmemBytes = pair_smem<MODE>();
+  lc.blockDim = dim3(PC::THREADS);
+  lc.dynamicSmemBytes = PC::SMEM;
   lc.stream = st;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -892,16 +904,19 @@ cudaError_t launch_pair(const Batch &bt, const TmapSet &tm, long long tiles, int
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   lc.attrs = attr;
   lc.numAttrs = pdl ? 2 : 1;
-  return cudaLaunchKernelEx(&lc, k_tiles_pair<MODE>, bt, tm, kept_rows);
+  return cudaLaunchKernelEx(&lc, k_tiles_pair<MODE, EW>, bt, tm, kept_rows);
 }
 
-template <int MODE> cudaError_t pair_configure() {
-  cudaError_t e = cudaFuncSetAttribute(k_tiles_pair<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pair_smem<MODE>());
+// can clusters of two CTAs of this kernel be launched at all?
+template <int MODE, int EW> cudaError_t pair_configure(bool &ok) {
+  using PC = PairCfg<MODE, EW>;
+  ok = false;
+  cudaError_t e = cudaFuncSetAttribute(k_tiles_pair<MODE, EW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PC::SMEM);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3(2);
-  lc.blockDim = dim3(THREADS);
-  lc.dynamicSmemBytes = pair_smem<MODE>();
+  lc.blockDim = dim3(PC::THREADS);
+  lc.dynamicSmemBytes = PC::SMEM;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
@@ -910,8 +925,9 @@ template <int MODE> cudaError_t pair_configure() {
   lc.attrs = attr;
   lc.numAttrs = 1;
   int n = 0;
-  e = cudaOccupancyMaxActiveClusters(&n, k_tiles_pair<MODE>, &lc);
-  if (e != cudaSuccess || n < 1) { (void)cudaGetLastError(); g_pair_ok = false; }
+  e = cudaOccupancyMaxActiveClusters(&n, k_tiles_pair<MODE, EW>, &lc);
+  if (e != cudaSuccess || n < 1) (void)cudaGetLastError();
+  else ok = true;
   return cudaSuccess;
 }
 }  // namespace
@@ -932,8 +948,9 @@ cudaError_t umma_configure() {
   e = cudaFuncSetAttribute(k_tiles_umma<MODE_ASSIGN, kWideBN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)TileCfg<kWideBN>::SMEM);
   if (e != cudaSuccess) return e;
-  g_pair_ok = true;
-  return pair_configure<MODE_SPREAD>();
+  e = pair_configure<MODE_GRAM, 16>(g_pair_gram_ok);
+  if (e != cudaSuccess) return e;
+  return pair_configure<MODE_SPREAD, 8>(g_pair_ok);
 }
 
 static int umma_grid_x(long long tiles, int B, int sms) {
@@ -943,12 +960,21 @@ static int umma_grid_x(long long tiles, int B, int sms) {
   return (int)(x < 1 ? 1 : x);
 }
 
-cudaError_t launch_gram_umma(const Batch &bt, int maxN, const ClusterCfg &cfg, cudaStream_t st) {
+cudaError_t launch_gram_umma(const Batch &bt, int maxN, const ClusterCfg &cfg, cudaStream_t st, int est_rows) {
   TmapSet tm;
   for (int b = 0; b < bt.B; ++b) {
     const ImgDesc &im = bt.img[b];
     if (!encode_rows(&tm.a[b], im.Kp, im.Np, bt.d_k, bt.d_k)) return cudaErrorInvalidValue;
     tm.b[b] = tm.a[b];
+  }
+  // With many blocks per SM (batches, long images) pairs of CTAs on 256 x 256 tiles with 16 epilogue warps each are
+  // faster: half the operand bytes per pair of blocks and a shorter epilogue.  With few (three per SM on one
+  // 7290-token image) the coarser tiles cost a round, and single CTAs on 128 x 128 blocks are.
+  if (est_rows < 1 || est_rows > maxN) est_rows = maxN;
+  const long long nq = (est_rows + BM - 1) / BM;
+  if (g_pair_gram_ok && nq * (nq + 1) / 2 * bt.B >= 6LL * cfg.sm_count) {
+    const long long n2 = (maxN + 2 * BM - 1) / (2 * BM);
+    return launch_pair<MODE_GRAM, 16>(bt, tm, n2 * (n2 + 1) / 2, 0, cfg, true, st);
   }
   const long long nb = (maxN + BM - 1) / BM;
   dim3 grid(umma_grid_x(nb * (nb + 1) / 2, bt.B, cfg.sm_count), bt.B);
@@ -979,7 +1005,7 @@ cudaError_t launch_spread_umma(const Batch &bt, int maxN, const ClusterCfg &cfg,
   }
   if (g_pair_ok) {
     const long long ptiles = (long long)((maxN + 2 * BM - 1) / (2 * BM)) * ((maxN + PBN - 1) / PBN);
-    return launch_pair<MODE_SPREAD>(bt, tm, ptiles, 0, cfg, false, st);
+    return launch_pair<MODE_SPREAD, 8>(bt, tm, ptiles, 0, cfg, false, st);
   }
   const long long tiles = (long long)((maxN + BM - 1) / BM) * ((maxN + kWideBN - 1) / kWideBN);
   dim3 grid(umma_grid_x(tiles, bt.B, cfg.sm_count), bt.B);

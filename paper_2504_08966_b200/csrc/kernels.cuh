@@ -86,7 +86,8 @@ void launch_spread_finish(const Batch &bt, float *max_dist, int32_t *layer_out, 
 // gram_umma.cu: tcgen05 versions of the two tile passes for bf16 keys whose width is a multiple of 64
 cudaError_t umma_configure();
 bool umma_supported(int d_k);
-cudaError_t launch_gram_umma(const Batch &bt, int maxN, const ClusterCfg &cfg, cudaStream_t st);
+// est_rows: an upper estimate of the survivors per image when the host has one (0: maxN)
+cudaError_t launch_gram_umma(const Batch &bt, int maxN, const ClusterCfg &cfg, cudaStream_t st, int est_rows = 0);
 cudaError_t launch_assign_umma(const Batch &bt, int maxN, bool kept_rows, const ClusterCfg &cfg, cudaStream_t st, bool labels = false);
 cudaError_t launch_members(const Batch &bt, int maxN, cudaStream_t st);
 cudaError_t launch_spread_umma(const Batch &bt, int maxN, const ClusterCfg &cfg, cudaStream_t st);
