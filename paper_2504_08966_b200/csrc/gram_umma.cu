@@ -703,20 +703,22 @@ template <int EW> struct SharedPair {
   __align__(16) float rn_col[EW][128];
 };
 
-// grid (2 P, B) in clusters of two CTAs along x, 64 + 32 EW threads, dynamic smem = PairCfg<MODE, EW>::SMEM.
-// Pair p takes the 256 x 256 tiles p, p + P, ... of the pass; CTA r of the pair owns the 128-row block 2 I + r of
-// tile (I, J).  In the all-pairs pass a tile is wanted when J >= I, and of the tile (I, I) the block (2 I + 1, 2 I)
-// lies below the diagonal and is computed but not used.
+// grid (2 P) in clusters of two CTAs, 64 + 32 EW threads, dynamic smem = PairCfg<MODE, EW>::SMEM.
+// The 256 x 256 tiles of all images (or layers) of the batch form one list, image after image; pair p takes the
+// items p, p + P, ... of it, so that the pairs stay equally loaded whatever the number of images.  CTA r of the
+// pair owns the 128-row block 2 I + r of tile (I, J).  In the all-pairs and largest-distance passes the tiles
+// with J >= I are listed, and of the tile (I, I) the block (2 I + 1, 2 I) lies below the diagonal: computed, not used.
 template <int MODE, int EW>
 __global__ void __launch_bounds__(PairCfg<MODE, EW>::THREADS, 1) k_tiles_pair(const __grid_constant__ Batch bt,
                                                                               const __grid_constant__ TmapSet tm, int kept_rows) {
   using PC = PairCfg<MODE, EW>;
   constexpr int PSTAGES = PC::STAGES;
   constexpr size_t PRING = PC::RING;
-  const ImgDesc &im = bt.img[blockIdx.y];
-  TL_SCOPE(im, MODE == MODE_GRAM ? 4 : 6);
+  constexpr int LIST = MODE == MODE_ASSIGN ? MODE_ASSIGN : MODE_GRAM;   // how the tiles of an image are listed
+  TL_SCOPE(bt.img[0], MODE == MODE_GRAM ? 4 : 6);
   extern __shared__ uint8_t smem_raw[];
   __shared__ SharedPair<EW> sh;
+  __shared__ int s_first[kMaxBatchPerLaunch + 1], s_rows[kMaxBatchPerLaunch], s_cols[kMaxBatchPerLaunch];
   uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_rank();
@@ -738,34 +740,52 @@ __global__ void __launch_bounds__(PairCfg<MODE, EW>::THREADS, 1) k_tiles_pair(co
   pdl_wait();
   pdl_trigger();
 
-  int nrows, ncols;
-  if (MODE == MODE_GRAM) { nrows = *im.q_ptr; ncols = nrows; }
-  else if (MODE == MODE_SPREAD) { nrows = im.N; ncols = im.N; }
-  else { nrows = (kept_rows & 1) ? *im.q_ptr : im.N; ncols = *im.C_ptr; }
-  const int nti = (nrows + 2 * BM - 1) / (2 * BM), ntj = (ncols + PBN - 1) / PBN;
-  const int ntiles = tile_count<MODE>(nti, ntj);
+  // rows, columns and first list position of every image
+  if (threadIdx.x == 0) {
+    int first = 0;
+    for (int b = 0; b < bt.B; ++b) {
+      const ImgDesc &ib = bt.img[b];
+      int nr, nc;
+      if (MODE == MODE_GRAM) { nr = *ib.q_ptr; nc = nr; }
+      else if (MODE == MODE_SPREAD) { nr = ib.N; nc = ib.N; }
+      else { nr = (kept_rows & 1) ? *ib.q_ptr : ib.N; nc = *ib.C_ptr; }
+      s_rows[b] = nr;
+      s_cols[b] = nc;
+      s_first[b] = first;
+      first += tile_count<LIST>((nr + 2 * BM - 1) / (2 * BM), (nc + PBN - 1) / PBN);
+    }
+    s_first[bt.B] = first;
+  }
+  __syncthreads();
+  const int total = s_first[bt.B];
   const int P = gridDim.x >> 1, pr = blockIdx.x >> 1;
   const int nslab = bt.d_k / BK;
-  auto wanted = [&](int I, int J) { return MODE != MODE_SPREAD || J >= I; };
+  // item -> image b (items only grow, so b only moves forward), tile (I, J), rows and columns of the image
+  auto locate = [&](int item, int &b, int &I, int &J, int &nrows, int &ncols) {
+    while (item >= s_first[b + 1]) ++b;
+    nrows = s_rows[b];
+    ncols = s_cols[b];
+    tile_at<LIST>(item - s_first[b], (nrows + 2 * BM - 1) / (2 * BM), (ncols + PBN - 1) / PBN, I, J);
+  };
   // columns the MMA has to produce: the rows x centres pass stops at the last centre, in steps of 32
-  auto width = [&](int J) {
+  auto width = [&](int J, int ncols) {
     if (MODE != MODE_ASSIGN) return PBN;
     const int left = ncols - J * PBN;
     return left >= PBN ? PBN : ((left + 31) & ~31);
   };
 
-  if (pr >= ntiles) {
+  if (pr >= total) {
   } else if (warp == 0) {
     // ---------------- TMA producer (each CTA for its own shared memory) ----------------
     if (lane == 0) {
-      const CUtensorMap *ma = &tm.a[blockIdx.y], *mb = &tm.b[blockIdx.y];
       uint32_t it = 0;
       bool ok = true;
-      for (int tile = pr; ok && tile < ntiles; tile += P) {
-        int I, J;
-        tile_at<MODE>(tile, nti, ntj, I, J);
-        if (!wanted(I, J)) continue;
-        const int bw = width(J);
+      int b = 0;
+      for (int item = pr; ok && item < total; item += P) {
+        int I, J, nrows, ncols;
+        locate(item, b, I, J, nrows, ncols);
+        const CUtensorMap *ma = &tm.a[b], *mb = &tm.b[b];
+        const int bw = width(J, ncols);
         for (int ks = 0; ks < nslab; ++ks, ++it) {
           const int s = it % PSTAGES;
           if (!mbar_wait(&sh.empty[s], ((it / PSTAGES) & 1) ^ 1)) { ok = false; break; }
@@ -783,16 +803,16 @@ __global__ void __launch_bounds__(PairCfg<MODE, EW>::THREADS, 1) k_tiles_pair(co
     if (lane == 0 && leader) {
       uint32_t it = 0, tcount = 0;
       bool ok = true;
-      for (int tile = pr; ok && tile < ntiles; tile += P) {
-        int I, J;
-        tile_at<MODE>(tile, nti, ntj, I, J);
-        if (!wanted(I, J)) continue;
+      int b = 0;
+      for (int item = pr; ok && item < total; item += P) {
+        int I, J, nrows, ncols;
+        locate(item, b, I, J, nrows, ncols);
         const uint32_t a = tcount % PNACC;
         if (!mbar_wait(&sh.acc_empty[a], ((tcount / PNACC) & 1) ^ 1)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + a * PBN;
         // kind::f16, fp32 accumulate, bf16 x bf16, both operands K-major, M = 256 over the pair, N = this tile's width
-        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(width(J) >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
+        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(width(J, ncols) >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
         for (int ks = 0; ks < nslab; ++ks, ++it) {
           const int s = it % PSTAGES;
           if (!mbar_wait(&sh.full[s], (it / PSTAGES) & 1)) { ok = false; break; }
@@ -819,31 +839,35 @@ __global__ void __launch_bounds__(PairCfg<MODE, EW>::THREADS, 1) k_tiles_pair(co
     float *rn_col = sh.rn_col[ew];
     uint32_t *tr = reinterpret_cast<uint32_t *>(ring + PRING - 1024) + ew * (32 * 36);   // all-pairs pass only
     uint32_t tcount = 0;
-    int band = 0;
     bool ok = true;
-    float mx = 0.f;
+    float mx = 0.f;                                 // largest distance of the current image (layer)
+    int b = 0, b_mx = 0;
     unsigned long long unused_seen = 0ull;
-    for (int tile = pr; ok && tile < ntiles; tile += P) {
-      int I, J;
-      tile_at<MODE>(tile, nti, ntj, I, J);
-      if (!wanted(I, J)) continue;
+    auto flush_mx = [&](int bb) {
+      const unsigned w = __reduce_max_sync(0xffffffffu, __float_as_uint(mx));
+      if (lane == 0 && w) atomicMax(reinterpret_cast<unsigned *>(&bt.img[bb].cnt[kCntSpread]), w);
+      mx = 0.f;
+    };
+    for (int item = pr; ok && item < total; item += P) {
+      int I, J, nrows, ncols;
+      locate(item, b, I, J, nrows, ncols);
+      if (MODE == MODE_SPREAD && b != b_mx) { flush_mx(b_mx); b_mx = b; }
+      const ImgDesc &im = bt.img[b];
       const uint32_t a = tcount % PNACC;
       const int R = 2 * I + (int)rank;              // this CTA's 128-row block
       const int cbase = J * PBN + half * PC::COLS;  // this warp's columns
-      const bool skip = MODE == MODE_GRAM && cbase / BM < R;   // below the diagonal
+      const bool skip = MODE != MODE_ASSIGN && cbase / BM < R;   // below the diagonal
       const uint32_t taddr = tmem_base + a * PBN + half * PC::COLS + ((uint32_t)(qd * 32) << 16);
       const uint32_t rel = map_to_rank(smem_u32(&sh.acc_empty[a]), 0);
+      int band = 0;
       ok = epi_tile<MODE, PC::COLS>(im, kept_rows, R, cbase, skip, nrows, ncols, taddr, &sh.acc_full[a], (tcount / PNACC) & 1,
-                               rn_col, tr, lane, qd, band, mx, [&]() { mbar_arrive_remote(rel); }, unused_seen);
+                                    rn_col, tr, lane, qd, band, mx, [&]() { mbar_arrive_remote(rel); }, unused_seen);
+      if (MODE == MODE_GRAM && band) atomicAdd(&im.cnt[PACT_CNT_BAND_DC], band);
       if (!ok) break;
       ++tcount;
     }
     if (!ok) atomicExch(&sh.abort, 1);
-    if (MODE == MODE_GRAM && band) atomicAdd(&im.cnt[PACT_CNT_BAND_DC], band);
-    if (MODE == MODE_SPREAD) {
-      const unsigned w = __reduce_max_sync(0xffffffffu, __float_as_uint(mx));
-      if (lane == 0 && w) atomicMax(reinterpret_cast<unsigned *>(&im.cnt[kCntSpread]), w);
-    }
+    if (MODE == MODE_SPREAD) flush_mx(b_mx);
   }
 
   tc_fence_before();
@@ -851,7 +875,8 @@ __global__ void __launch_bounds__(PairCfg<MODE, EW>::THREADS, 1) k_tiles_pair(co
   cluster_barrier();                                  // nothing is in flight towards the other CTA any more
   tc_fence_after();
   if (warp == 1) tmem_dealloc2(tmem_base, TMEM_COLS);
-  if (threadIdx.x == 0 && sh.abort) atomicMin(&im.cnt[PACT_CNT_STATUS], (int)PACT_ERR_TIMEOUT);
+  if (threadIdx.x == 0 && sh.abort)
+    for (int b = 0; b < bt.B; ++b) atomicMin(&bt.img[b].cnt[PACT_CNT_STATUS], (int)PACT_ERR_TIMEOUT);
 }
 
 // ---- host side -----------------------------------------------------------------------------------
@@ -887,11 +912,11 @@ template <int MODE, int EW>
 cudaError_t launch_pair(const Batch &bt, const TmapSet &tm, long long tiles, int kept_rows, const ClusterCfg &cfg, bool pdl,
                         cudaStream_t st) {
   using PC = PairCfg<MODE, EW>;
-  long long P = cfg.sm_count / 2 / bt.B;              // one pair per two SMs: all pairs of the batch run at once
-  if (P > tiles) P = tiles;
+  long long P = cfg.sm_count / 2;                     // one pair per two SMs
+  if (P > tiles * bt.B) P = tiles * bt.B;
   if (P < 1) P = 1;
   cudaLaunchConfig_t lc = {};
-  lc.gridDim = dim3((unsigned)(2 * P), bt.B);
+  lc.gridDim = dim3((unsigned)(2 * P));
   lc.blockDim = dim3(PC::THREADS);
   lc.dynamicSmemBytes = PC::SMEM;
   lc.stream = st;
