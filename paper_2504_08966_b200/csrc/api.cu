@@ -565,16 +565,19 @@ pact_status pact_reduce(pact_ctx *ctx, const pact_image *imgs, int B, const pact
     else launch_gram(bt, cmaxN, bf, ctx->ccfg, st);
     CK(mark());
     CK(launch_centers(bt, cmaxQ, bf, ctx->ccfg, ctx->sweep_limit, st));  CK(mark());
-    // on the tensor-core path the labels and member counts are formed as the rows x centres pass finishes
-    // groups of rows, and one kernel places the members; otherwise k_lists does both
-    if (ctx->umma) CK(launch_assign_umma(bt, cmaxN, false, ctx->ccfg, st, true));
+    // On the tensor-core path with little work per SM (one image) the labels and member counts are formed as
+    // the rows x centres pass finishes groups of rows, and one kernel places the members.  With much work per SM
+    // the pass runs on pairs of CTAs, and k_lists forms labels and lists as it does on the fp32 path.
+    const bool pairs = ctx->umma && umma_pairs_for_assign(cmaxN, nb, ctx->ccfg);
+    const bool fused_labels = ctx->umma && !pairs;
+    if (ctx->umma) CK(launch_assign_umma(bt, cmaxN, false, ctx->ccfg, st, fused_labels, pairs));
     else launch_assign(bt, cmaxN, bf, ROWS_ALL, ctx->ccfg, st);
     CK(mark());
-    if (ctx->umma) CK(launch_members(bt, cmaxN, st));
+    if (fused_labels) CK(launch_members(bt, cmaxN, st));
     else CK(launch_lists(bt, cmaxN, bf, true, ctx->spin_limit, st));
     CK(mark());
     CK(launch_merge(bt, bf, ctx->out == PACT_BF16, ctx->ccfg, st));  CK(mark());
-    ctx->launches += euti_kernels(0) + 4 + (ctx->umma ? 1 : lists_kernels(cmaxN, nb));
+    ctx->launches += euti_kernels(0) + 4 + (fused_labels ? 1 : lists_kernels(cmaxN, nb));
     CK(cudaGetLastError());
     for (int b = 0; b < nb; ++b)
       CK(cudaMemcpyAsync(bt.img[b].counters_user, bt.img[b].cnt, PACT_N_COUNTERS * sizeof(int32_t),

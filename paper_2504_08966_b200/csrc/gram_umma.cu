@@ -626,8 +626,8 @@ __global__ void __launch_bounds__(THREADS, 1) k_tiles_umma(const __grid_constant
 // columns (half of operand B), CTA 0 issues tcgen05.mma.cta_group::2 for both, and each CTA finds its
 // 128 x 256 part of the product in its own tensor memory.  A CTA therefore fetches half as many operand
 // bytes from the L2 per output element as it does alone.  The largest-distance pass always runs this way, the
-// all-pairs pass when an SM has six or more 128 x 128 blocks to do (with fewer, the coarser tiles cost a round);
-// the rows x centres pass measured slower this way.
+// all-pairs pass when an SM has six or more 128 x 128 blocks to do and the rows x centres pass when it has two or
+// more 128-row blocks (with fewer, the coarser tiles cost a round).
 //   full[s]      in CTA 0: both CTAs' copies of stage s report their bytes there
 //   empty[s]     in each CTA: tcgen05.commit (multicast to both CTAs) once the MMAs have read stage s
 //   acc_full[a]  in each CTA: tcgen05.commit (multicast) once accumulator a is complete
@@ -907,6 +907,7 @@ bool umma_supported(int d_k) { return g_encode != nullptr && d_k % BK == 0; }
 namespace {
 bool g_pair_ok = false;                               // clusters of two CTAs of the pair kernel can be launched
 bool g_pair_gram_ok = false;                          // ... of its all-pairs form with 16 epilogue warps
+bool g_pair_assign_ok = false;                        // ... of its rows x centres form
 
 template <int MODE, int EW>
 cudaError_t launch_pair(const Batch &bt, const TmapSet &tm, long long tiles, int kept_rows, const ClusterCfg &cfg, bool pdl,
@@ -973,6 +974,8 @@ cudaError_t umma_configure() {
   e = cudaFuncSetAttribute(k_tiles_umma<MODE_ASSIGN, kWideBN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)TileCfg<kWideBN>::SMEM);
   if (e != cudaSuccess) return e;
+  e = pair_configure<MODE_ASSIGN, 8>(g_pair_assign_ok);
+  if (e != cudaSuccess) return e;
   e = pair_configure<MODE_GRAM, 16>(g_pair_gram_ok);
   if (e != cudaSuccess) return e;
   return pair_configure<MODE_SPREAD, 8>(g_pair_ok);
@@ -1006,7 +1009,16 @@ cudaError_t launch_gram_umma(const Batch &bt, int maxN, const ClusterCfg &cfg, c
   return launch_k(k_tiles_umma<MODE_GRAM, kGramBN>, grid, dim3(THREADS), TileCfg<kGramBN>::SMEM, st, true, bt, tm, 0);
 }
 
-cudaError_t launch_assign_umma(const Batch &bt, int maxN, bool kept_rows, const ClusterCfg &cfg, cudaStream_t st, bool labels) {
+bool umma_pairs_for_assign(int maxN, int B, const ClusterCfg &cfg) {
+  // with two or more 128-row blocks per SM (batches, long images) pairs of CTAs on 256 x 256 tiles are faster:
+  // the pass is bound by operand bytes from the L2, and a pair fetches two thirds of them
+  return g_pair_assign_ok && (long long)((maxN + BM - 1) / BM) * B >= 2LL * cfg.sm_count;
+}
+
+// labels: the single-CTA kernel also forms labels and member counts (all-token rows only); pairs: the pair kernel
+// (all-token rows, no labels)
+cudaError_t launch_assign_umma(const Batch &bt, int maxN, bool kept_rows, const ClusterCfg &cfg, cudaStream_t st, bool labels,
+                               bool pairs) {
   TmapSet tm;
   for (int b = 0; b < bt.B; ++b) {
     const ImgDesc &im = bt.img[b];
@@ -1014,6 +1026,10 @@ cudaError_t launch_assign_umma(const Batch &bt, int maxN, bool kept_rows, const 
       if (!encode_rows(&tm.a[b], im.Kp, im.Np, bt.d_k, bt.d_k)) return cudaErrorInvalidValue;
     } else if (!encode_rows(&tm.a[b], im.Kc, im.N, im.ldKc, bt.d_k)) return cudaErrorInvalidValue;
     if (!encode_rows(&tm.b[b], im.Kcen, im.Np, bt.d_k, bt.d_k)) return cudaErrorInvalidValue;
+  }
+  if (pairs && !kept_rows && g_pair_assign_ok) {
+    const long long pt = (long long)((maxN + 2 * BM - 1) / (2 * BM)) * ((maxN + PBN - 1) / PBN);
+    return launch_pair<MODE_ASSIGN, 8>(bt, tm, pt, 0, cfg, true, st);
   }
   const long long tiles = (long long)((maxN + BM - 1) / BM) * ((maxN + kWideBN - 1) / kWideBN);
   dim3 grid(umma_grid_x(tiles, bt.B, cfg.sm_count), bt.B);

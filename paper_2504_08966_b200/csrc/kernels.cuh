@@ -88,7 +88,9 @@ cudaError_t umma_configure();
 bool umma_supported(int d_k);
 // est_rows: an upper estimate of the survivors per image when the host has one (0: maxN)
 cudaError_t launch_gram_umma(const Batch &bt, int maxN, const ClusterCfg &cfg, cudaStream_t st, int est_rows = 0);
-cudaError_t launch_assign_umma(const Batch &bt, int maxN, bool kept_rows, const ClusterCfg &cfg, cudaStream_t st, bool labels = false);
+cudaError_t launch_assign_umma(const Batch &bt, int maxN, bool kept_rows, const ClusterCfg &cfg, cudaStream_t st, bool labels = false,
+                               bool pairs = false);
+bool umma_pairs_for_assign(int maxN, int B, const ClusterCfg &cfg);
 cudaError_t launch_members(const Batch &bt, int maxN, cudaStream_t st);
 cudaError_t launch_spread_umma(const Batch &bt, int maxN, const ClusterCfg &cfg, cudaStream_t st);
 
