@@ -1,4 +1,4 @@
-// mbarrier and bulk-copy (TMA) primitives shared by the kernels that stage data through shared memory.
+// mbarrier primitives of the kernels that stage data through shared memory with tiled bulk copies (TMA).
 // Every wait is bounded: after kWaitNs of wall time it returns false and the caller gives up cleanly.
 #pragma once
 #include <stdint.h>
@@ -52,12 +52,6 @@ __device__ __forceinline__ bool mbar_wait_warp(uint64_t *bar, uint32_t parity) {
   int ok = 1;
   if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity) ? 1 : 0;
   return __shfl_sync(0xffffffffu, ok, 0) != 0;
-}
-
-// Plain (untiled) bulk copy global -> shared: both addresses 16-byte aligned, bytes a multiple of 16.
-__device__ __forceinline__ void bulk_load_1d(void *dst, const void *src, uint32_t bytes, uint64_t *bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
 }  // namespace pact
