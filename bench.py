@@ -188,6 +188,49 @@ def reference_arm(args):
     print(json.dumps(line))
 
 
+def other_workload(name, steps=100):
+    """Step time of one of the other synthetic workloads (graph replay, rotating input copies), measured in the
+    same process as the headline so that one run times them all."""
+    from paper_2504_08966_b200 import binding as pb
+    from paper_2504_08966_b200 import workloads
+    wl = workloads.build(name, seed={"video": 3, "batched": 2, "stress": 4}[name])
+    ctx = pb.Context(wl.d, wl.n_qh, wl.n_kvh, wl.d_h, wl.dtype, torch.bfloat16)
+    params = pb.make_params(lam=wl.lam, d_c=wl.d_c, d_n=wl.d_n, alpha=wl.alpha)
+    in_bytes = sum(im.H.numel() * 2 + im.K.numel() * 2 + im.Q.numel() * 2 + im.P.numel() * 4 for im in wl.images)
+    copies = max(2, min(4, int(4e9 // in_bytes)))
+    sets = [[pb.device_image(img, torch.bfloat16) for img in wl.images] for _ in range(copies)]
+    B = len(wl.images)
+    ctx.ensure_workspace(B, max(im.N for im in wl.images))
+    graphs = [ctx.pact_graph_create(ims, params) for ims in sets]
+    for i in range(6):
+        graphs[i % copies].launch()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        graphs[i % copies].launch()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    pk = _peaks()
+    bytes_, flops, status = 0.0, 0.0, 0
+    for img, im in zip(wl.images, sets[(steps - 1) % copies]):
+        cnt = im.counters.cpu().numpy()
+        q, Cn = int(cnt[pb.CNT["q"]]), int(cnt[pb.CNT["C"]])
+        status = min(status, int(cnt[pb.CNT["status"]]))
+        T = img.n_total - img.N
+        bytes_ += (img.N * wl.d * 2 + img.N * wl.d_k * 2 + img.N * wl.n_qh * wl.d_h * 2 + 4 * img.n_total + 2 * T * wl.d * 2
+                   + Cn * (wl.d * 2 + 8) + 4 * img.N)
+        flops += 2.0 * wl.d_k * (q * (q + 1) / 2) + 2.0 * wl.d_k * img.N * Cn
+    t_roof = max(bytes_ / (pk["hbm_gbs"] * 1e9), flops / (pk["bf16_tflops"] * 1e12))
+    n_vis = sum(im.N for im in wl.images)
+    for g in graphs:
+        g.close()
+    return {"images": B, "N": wl.images[0].N, "steps": steps, "ms_per_step": ms, "value": n_vis / (ms * 1e-3), "unit": UNIT,
+            "t_roof_us": t_roof * 1e6, "roofline_path_frac": t_roof / (ms * 1e-3), "status": status,
+            "l2": f"{copies} input copies rotated"}
+
+
 STAGE_WORKLOADS = ("euti_only", "dbdpc_only", "layer_choice")
 
 
@@ -323,6 +366,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="pact", choices=["pact", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-other-workloads", action="store_true",
+                    help="skip the video / batched / stress step times that the single_image line carries along")
     ap.add_argument("--in-flight", type=int, default=4,
                     help="also report the throughput with this many independent single-image requests in flight")
     ap.add_argument("--workload", default="single_image",
@@ -574,6 +619,8 @@ def main():
                               "alg_flops": per_img_flops * B, "peak_source": pk["source"]},
             "stages_us": stages_us,
         }
+        if world == 1 and args.workload == "single_image" and not args.no_other_workloads:
+            line["other_workloads"] = {w: other_workload(w) for w in ("video", "batched", "stress")}
         if not args.no_cpu_baseline and world == 1:
             step(0)                                # outputs of input copy 0 as the timed launch leaves them
             torch.cuda.synchronize()
